@@ -1,0 +1,159 @@
+/*
+ * kvh.h — C ABI of the per-chunk KV-cache codec (CUDA, sm_100a).
+ *
+ * The codec is the executor's data path in the paper's design (Design
+ * section: estimator, policy optimizer, executor): it stores a context's KV
+ * tensors at the quality the policy chose ("evict, store in full quality or
+ * compress", last paragraph of the Design section) and, on a cache hit,
+ * decompresses a stored chunk into the serving engine's paged bf16 KV (the
+ * "decompression overhead" the estimator profiles).  A KV tensor is l layers
+ * x {K,V} x N tokens x c channels of bf16 (the paper's N, c, l); a quality
+ * level k is one rung of the ladder below.
+ *
+ * Levels (the paper prints only "2 bits" and "full quality"; the ladder, the
+ * group geometry and the byte format are this library's definition):
+ *   0  raw bf16, lossless                      16 bits/element
+ *   1  8-bit asymmetric group quantisation      9 bits/element
+ *   2  4-bit                                    5 bits/element
+ *   3  2-bit                                    3 bits/element
+ * K groups: one channel over 32 consecutive tokens of a chunk.  V groups: 32
+ * consecutive channels of one token.  Per group a u32 = bf16(min) |
+ * bf16(max) << 16.  A chunk is at most 256 tokens; its stream is, per layer,
+ * Kmeta | Kcodes | Vmeta | Vcodes, each zero-padded to 128 bytes, with
+ * Kmeta[ceil(n/32)][c], Vmeta[n][c/32], and the code of element (t, ch) in
+ * bits [b*(t*c+ch), +b) of its section read as a little-endian bit string.
+ * Level 0 has no metadata; its code sections are the bf16 rows themselves.
+ * Arithmetic, binary32 round-to-nearest-even: r = max - min; when
+ * 2^-100 <= r <= FLT_MAX, inv = qmax / r and scale = r / qmax, otherwise both
+ * are 0 (every code 0, decodes to min); q = clamp(rint((x - min) * inv), 0,
+ * qmax); xhat = bf16_rne(fma(q, scale, min)).  Inputs must be finite.
+ *
+ * Conventions.  Pointers marked [device] are CUDA device pointers, [host]
+ * host pointers.  The caller owns every buffer; the library allocates no
+ * device memory and keeps no state between calls.  Device work is enqueued on
+ * `stream` (a cudaStream_t passed as void*, NULL = the default stream) and
+ * the call returns without waiting.  Argument errors are reported by the
+ * return value with nothing enqueued.  Errors only the GPU can see (a page id
+ * outside the pool, a descriptor that does not fit its buffer) make the
+ * kernel skip the offending chunk or page and atomicMax the status code into
+ * *dev_status [device, may be NULL]; nothing traps.  No CPU fallback exists.
+ */
+#ifndef KVH_H
+#define KVH_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVH_FORMAT_VERSION 1
+#define KVH_CHUNK_TOKENS 256   /* most tokens in one chunk */
+#define KVH_GROUP 32           /* tokens per K group, channels per V group */
+#define KVH_SECTION_ALIGN 128  /* every section and chunk starts on this boundary */
+
+typedef int kvh_status;
+enum {
+    KVH_OK = 0,
+    KVH_ERR_INVALID_ARG = 1,      /* NULL pointer, negative count */
+    KVH_ERR_BAD_LEVEL = 2,        /* level outside 0..3 */
+    KVH_ERR_BAD_SHAPE = 3,        /* c not a multiple of 32, n_tok outside 1..256, ... */
+    KVH_ERR_MISALIGNED = 4,       /* base not 128-byte (streams) / 16-byte (KV, pool) aligned */
+    KVH_ERR_BUFFER_TOO_SMALL = 5, /* stream or page table shorter than a descriptor needs */
+    KVH_ERR_PAGE_OOB = 6,         /* page id outside [0, num_pages): device-reported */
+    KVH_ERR_CUDA = 7,             /* a CUDA runtime call failed (launch error) */
+    KVH_ERR_TIMEOUT = 8           /* reserved: a bounded device wait ran out */
+};
+
+/* The serving engine's paged KV pool: element (layer, kv, page, slot, ch) is at
+ * base + layer*layer_stride + kv*kv_stride + page*page_stride + slot*n_channels
+ * + ch, in bf16 elements.  Strides must be multiples of 8 elements. */
+typedef struct {
+    void *base;            /* [device] bf16 */
+    int64_t layer_stride;
+    int64_t kv_stride;     /* kv = 0 for K, 1 for V */
+    int64_t page_stride;
+    int32_t num_pages;
+    int32_t page_tokens;   /* tokens per page; must divide 256 (16 in the benchmark) */
+    int32_t n_layers;
+    int32_t n_channels;
+} kvh_pool;
+
+/* One stored chunk.  stream_off: byte offset of the chunk in the stream buffer
+ * (multiple of 128).  pt_off: index in the page table of the chunk's first
+ * page id (decode only); the chunk uses ceil(n_tok / page_tokens) entries. */
+typedef struct {
+    uint64_t stream_off;
+    int32_t level;
+    int32_t n_tok;
+    int32_t pt_off;
+    int32_t reserved;      /* must be 0 */
+} kvh_chunk_desc;
+
+int kvh_format_version(void);
+int kvh_num_levels(void);
+const char *kvh_status_string(kvh_status s);
+
+/* Properties of a level: code bits per element, group size, 1 if lossless.
+ * Any out pointer may be NULL.  [host] */
+kvh_status kvh_level_info(int level, int *bits, int *group, int *lossless);
+
+/* size(i, M, R) of the paper's utility definition for one chunk: bytes the
+ * stored form of n_tokens (1..256) tokens takes at `level`.  Pure host
+ * arithmetic.  *out [host]. */
+kvh_status kvh_level_bytes(int level, int n_layers, int n_channels, int n_tokens,
+                           uint64_t *out);
+
+/* Lay out a context of n_tokens as ceil(n_tokens/256) chunks.  chunk_levels
+ * [host, one entry per chunk] or NULL to use `level` for all.  Chunk i gets
+ * stream_off = stream_base + sum of the sizes before it, pt_off = pt_base +
+ * i * (256 / page_tokens).  descs_out [host, n chunks] may be NULL to ask only
+ * for *total_bytes [host] (bytes from stream_base to the end of the last chunk).
+ * Pure host arithmetic. */
+kvh_status kvh_plan_chunks(int n_layers, int n_channels, int64_t n_tokens,
+                           const int32_t *chunk_levels, int level,
+                           uint64_t stream_base, int32_t pt_base, int32_t page_tokens,
+                           kvh_chunk_desc *descs_out, uint64_t *total_bytes);
+
+/* Encode a whole context at one level (the per-entry decision (M_i, R_i) of
+ * the utility definition).  kv [device]: bf16 [n_layers][2][n_tokens][n_channels],
+ * contiguous, 16-byte aligned.  out [device]: 128-byte aligned, out_capacity
+ * bytes; chunk i lands at i * kvh_level_bytes(level, ..., 256).  Returns
+ * KVH_ERR_BUFFER_TOO_SMALL if the context does not fit. */
+kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                      int level, void *out, uint64_t out_capacity,
+                      int32_t *dev_status, void *stream);
+
+/* Encode a context with a level per chunk.  descs [device, n_chunks =
+ * ceil(n_tokens/256)]: desc i describes tokens [256 i, 256 i + n_tok) and where
+ * its stream goes (as laid out by kvh_plan_chunks).  A descriptor with a bad
+ * level, an n_tok that does not match the context, a misaligned offset or an
+ * extent beyond out_capacity is skipped and reported through *dev_status. */
+kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                             const kvh_chunk_desc *descs, int n_chunks,
+                             void *out, uint64_t out_capacity,
+                             int32_t *dev_status, void *stream);
+
+/* Decode one stored chunk (cache hit) into the pool.  chunk [device, 128-byte
+ * aligned]: the chunk's stream.  page_ids [device]: ceil(n_tok/page_tokens)
+ * page ids; token t goes to page page_ids[t / page_tokens], slot
+ * t % page_tokens, in every layer and for K and V alike.  Slots past n_tok in
+ * the last page are not written.  pool [host struct, device memory]. */
+kvh_status kvh_decode_to_pages(const void *chunk, int level, int n_tok,
+                               const int32_t *page_ids, const kvh_pool *pool,
+                               int32_t *dev_status, void *stream);
+
+/* Decode many stored chunks of mixed levels in one launch.  streams_base
+ * [device, 128-byte aligned, streams_bytes long]; descs [device, n_chunks];
+ * page_table [device, page_table_len entries].  Chunk i reads its stream at
+ * streams_base + descs[i].stream_off and its page ids at page_table +
+ * descs[i].pt_off.  Bad descriptors are skipped and reported. */
+kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes,
+                            const kvh_chunk_desc *descs, int n_chunks,
+                            const int32_t *page_table, int64_t page_table_len,
+                            const kvh_pool *pool, int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVH_H */

@@ -1,0 +1,11 @@
+"""B200-native per-chunk KV-cache codec: thin Python binding over the C ABI in include/kvh.h.
+
+Every step of the path runs in the CUDA kernels of ``libkvh.so``; this package
+only marshals arguments (tensor pointers, the current CUDA stream).  There is no
+CPU fallback: calling into the library without the built extension raises.
+"""
+from .binding import (  # noqa: F401
+    CHUNK_TOKENS, GROUP, NUM_LEVELS, ChunkDesc, KvhError, Pool, decode_batch, decode_to_pages,
+    descs_to_tensor, encode, encode_chunks, format_version, level_bytes, level_info, lib,
+    plan_chunks, status_string,
+)

@@ -1,0 +1,230 @@
+// Host side of the C ABI declared in include/kvh.h: argument validation, size
+// arithmetic and kernel launches.  No device memory is allocated here and no
+// state survives a call.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvh.h"
+#include "kvh_decode.cuh"
+#include "kvh_encode.cuh"
+#include "kvh_format.cuh"
+
+using namespace kvh;
+
+namespace {
+
+bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+kvh_status check_shape(int level, int l, int c)
+{
+    if (level < 0 || level >= kNumLevels) return KVH_ERR_BAD_LEVEL;
+    if (l <= 0 || c <= 0 || c % kGroup != 0) return KVH_ERR_BAD_SHAPE;
+    return KVH_OK;
+}
+
+kvh_status check_pool(const kvh_pool *pool)
+{
+    if (!pool || !pool->base) return KVH_ERR_INVALID_ARG;
+    if (pool->n_layers <= 0 || pool->n_channels <= 0 || pool->n_channels % kGroup != 0) return KVH_ERR_BAD_SHAPE;
+    if (pool->page_tokens <= 0 || kChunkTokens % pool->page_tokens != 0) return KVH_ERR_BAD_SHAPE;
+    if (pool->num_pages <= 0) return KVH_ERR_BAD_SHAPE;
+    if (pool->layer_stride < 0 || pool->kv_stride < 0 || pool->page_stride < 0) return KVH_ERR_BAD_SHAPE;
+    if (!aligned(pool->base, 16) || pool->layer_stride % 8 || pool->kv_stride % 8 || pool->page_stride % 8)
+        return KVH_ERR_MISALIGNED;
+    return KVH_OK;
+}
+
+// one CTA per (chunk, layer, K|V, tile); 0 if the grid would not fit
+unsigned grid_for(int64_t n_chunks, int l)
+{
+    const int64_t g = n_chunks * l * 2 * kTilesPerChunk;
+    return (g <= 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;
+}
+
+kvh_status launch_status()
+{
+    return cudaPeekAtLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;
+}
+
+kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, void *stream)
+{
+    p.pool = static_cast<uint16_t *>(pool->base);
+    p.layer_stride = pool->layer_stride;
+    p.kv_stride = pool->kv_stride;
+    p.page_stride = pool->page_stride;
+    p.num_pages = pool->num_pages;
+    p.page_tokens = pool->page_tokens;
+    p.l = pool->n_layers;
+    p.c = pool->n_channels;
+    const unsigned grid = grid_for(n_chunks, p.l);
+    if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+int kvh_format_version(void) { return KVH_FORMAT_VERSION; }
+int kvh_num_levels(void) { return kNumLevels; }
+
+const char *kvh_status_string(kvh_status s)
+{
+    switch (s) {
+    case KVH_OK: return "ok";
+    case KVH_ERR_INVALID_ARG: return "invalid argument";
+    case KVH_ERR_BAD_LEVEL: return "level outside 0..3";
+    case KVH_ERR_BAD_SHAPE: return "unsupported shape";
+    case KVH_ERR_MISALIGNED: return "misaligned pointer, offset or stride";
+    case KVH_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case KVH_ERR_PAGE_OOB: return "page id outside the pool";
+    case KVH_ERR_CUDA: return "CUDA runtime error";
+    case KVH_ERR_TIMEOUT: return "device wait timed out";
+    default: return "unknown status";
+    }
+}
+
+kvh_status kvh_level_info(int level, int *bits, int *group, int *lossless)
+{
+    if (level < 0 || level >= kNumLevels) return KVH_ERR_BAD_LEVEL;
+    if (bits) *bits = level_bits(level);
+    if (group) *group = level == 0 ? 0 : kGroup;
+    if (lossless) *lossless = level == 0;
+    return KVH_OK;
+}
+
+kvh_status kvh_level_bytes(int level, int n_layers, int n_channels, int n_tokens, uint64_t *out)
+{
+    if (!out) return KVH_ERR_INVALID_ARG;
+    const kvh_status s = check_shape(level, n_layers, n_channels);
+    if (s != KVH_OK) return s;
+    if (n_tokens < 1 || n_tokens > kChunkTokens) return KVH_ERR_BAD_SHAPE;
+    *out = chunk_bytes(level, n_layers, n_channels, n_tokens);
+    return KVH_OK;
+}
+
+kvh_status kvh_plan_chunks(int n_layers, int n_channels, int64_t n_tokens, const int32_t *chunk_levels,
+                           int level, uint64_t stream_base, int32_t pt_base, int32_t page_tokens,
+                           kvh_chunk_desc *descs_out, uint64_t *total_bytes)
+{
+    if (n_tokens <= 0 || pt_base < 0) return KVH_ERR_INVALID_ARG;
+    if (page_tokens <= 0 || kChunkTokens % page_tokens != 0) return KVH_ERR_BAD_SHAPE;
+    if (stream_base % KVH_SECTION_ALIGN) return KVH_ERR_MISALIGNED;
+    const int64_t n_chunks = (n_tokens + kChunkTokens - 1) / kChunkTokens;
+    const int64_t pages_per_chunk = kChunkTokens / page_tokens;
+    if (pt_base + n_chunks * pages_per_chunk > 0x7fffffffLL) return KVH_ERR_BAD_SHAPE;
+    uint64_t off = stream_base;
+    for (int64_t i = 0; i < n_chunks; ++i) {
+        const int k = chunk_levels ? chunk_levels[i] : level;
+        const kvh_status s = check_shape(k, n_layers, n_channels);
+        if (s != KVH_OK) return s;
+        const int64_t left = n_tokens - i * kChunkTokens;
+        const int n = (int)(left < kChunkTokens ? left : kChunkTokens);
+        if (descs_out) {
+            descs_out[i].stream_off = off;
+            descs_out[i].level = k;
+            descs_out[i].n_tok = n;
+            descs_out[i].pt_off = (int32_t)(pt_base + i * pages_per_chunk);
+            descs_out[i].reserved = 0;
+        }
+        off += chunk_bytes(k, n_layers, n_channels, n);
+    }
+    if (total_bytes) *total_bytes = off - stream_base;
+    return KVH_OK;
+}
+
+kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_channels, int level,
+                      void *out, uint64_t out_capacity, int32_t *dev_status, void *stream)
+{
+    if (!kv || !out || n_tokens <= 0) return KVH_ERR_INVALID_ARG;
+    const kvh_status s = check_shape(level, n_layers, n_channels);
+    if (s != KVH_OK) return s;
+    if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN)) return KVH_ERR_MISALIGNED;
+    uint64_t need = 0;
+    const kvh_status ps = kvh_plan_chunks(n_layers, n_channels, n_tokens, nullptr, level, 0, 0, 16, nullptr, &need);
+    if (ps != KVH_OK) return ps;
+    if (need > out_capacity) return KVH_ERR_BUFFER_TOO_SMALL;
+    const int64_t n_chunks = (n_tokens + kChunkTokens - 1) / kChunkTokens;
+    const unsigned grid = grid_for(n_chunks, n_layers);
+    if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    EncodeParams p{};
+    p.kv = static_cast<const uint16_t *>(kv);
+    p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+    p.descs = nullptr;
+    p.level = level;
+    p.full_chunk_bytes = chunk_bytes(level, n_layers, n_channels, kChunkTokens);
+    p.out = static_cast<uint8_t *>(out);
+    p.capacity = out_capacity;
+    p.status = dev_status;
+    encode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return launch_status();
+}
+
+kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                             const kvh_chunk_desc *descs, int n_chunks, void *out, uint64_t out_capacity,
+                             int32_t *dev_status, void *stream)
+{
+    if (!kv || !out || !descs || n_tokens <= 0) return KVH_ERR_INVALID_ARG;
+    const kvh_status s = check_shape(0, n_layers, n_channels);
+    if (s != KVH_OK) return s;
+    if ((int64_t)n_chunks != (n_tokens + kChunkTokens - 1) / kChunkTokens) return KVH_ERR_BAD_SHAPE;
+    if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
+    const unsigned grid = grid_for(n_chunks, n_layers);
+    if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    EncodeParams p{};
+    p.kv = static_cast<const uint16_t *>(kv);
+    p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+    p.descs = descs;
+    p.out = static_cast<uint8_t *>(out);
+    p.capacity = out_capacity;
+    p.status = dev_status;
+    encode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return launch_status();
+}
+
+kvh_status kvh_decode_to_pages(const void *chunk, int level, int n_tok, const int32_t *page_ids,
+                               const kvh_pool *pool, int32_t *dev_status, void *stream)
+{
+    if (!chunk || !page_ids) return KVH_ERR_INVALID_ARG;
+    const kvh_status ps = check_pool(pool);
+    if (ps != KVH_OK) return ps;
+    const kvh_status s = check_shape(level, pool->n_layers, pool->n_channels);
+    if (s != KVH_OK) return s;
+    if (n_tok < 1 || n_tok > kChunkTokens) return KVH_ERR_BAD_SHAPE;
+    if (!aligned(chunk, KVH_SECTION_ALIGN) || !aligned(page_ids, 4)) return KVH_ERR_MISALIGNED;
+    DecodeParams p{};
+    p.streams = static_cast<const uint8_t *>(chunk);
+    p.streams_bytes = chunk_bytes(level, pool->n_layers, pool->n_channels, n_tok);
+    p.descs = nullptr;
+    p.single.stream_off = 0;
+    p.single.level = level;
+    p.single.n_tok = n_tok;
+    p.single.pt_off = 0;
+    p.page_table = page_ids;
+    p.page_table_len = (n_tok + pool->page_tokens - 1) / pool->page_tokens;
+    p.status = dev_status;
+    return launch_decode(p, pool, 1, stream);
+}
+
+kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes, const kvh_chunk_desc *descs,
+                            int n_chunks, const int32_t *page_table, int64_t page_table_len,
+                            const kvh_pool *pool, int32_t *dev_status, void *stream)
+{
+    if (!streams_base || !descs || !page_table || n_chunks < 0 || page_table_len < 0) return KVH_ERR_INVALID_ARG;
+    const kvh_status ps = check_pool(pool);
+    if (ps != KVH_OK) return ps;
+    if (!aligned(streams_base, KVH_SECTION_ALIGN) || !aligned(descs, 8) || !aligned(page_table, 4))
+        return KVH_ERR_MISALIGNED;
+    if (n_chunks == 0) return KVH_OK;
+    DecodeParams p{};
+    p.streams = static_cast<const uint8_t *>(streams_base);
+    p.streams_bytes = streams_bytes;
+    p.descs = descs;
+    p.page_table = page_table;
+    p.page_table_len = page_table_len;
+    p.status = dev_status;
+    return launch_decode(p, pool, n_chunks, stream);
+}
+
+}  // extern "C"

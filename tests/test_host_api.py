@@ -1,0 +1,133 @@
+"""Host-side checks that need no GPU: the C-ABI library builds, loads and exports
+every symbol the header declares; the size and layout arithmetic agrees with the
+oracle; argument errors are reported without touching a device."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def kvh():
+    from paper_2509_00105_b200 import _build
+    _build.build()
+    import paper_2509_00105_b200 as k
+    k.lib()
+    return k
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "kvh.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kvh_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(kvh):
+    names = declared_symbols()
+    assert {"kvh_level_bytes", "kvh_encode", "kvh_decode_to_pages", "kvh_decode_batch"} <= set(names)
+    L = ctypes.CDLL(str(kvh.binding._LIB_PATH))
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_versions_and_level_info(kvh):
+    assert kvh.format_version() == 1
+    assert kvh.lib().kvh_num_levels() == 4
+    assert [kvh.level_info(k) for k in range(4)] == [(16, 0, True), (8, 32, False), (4, 32, False), (2, 32, False)]
+    with pytest.raises(kvh.KvhError) as e:
+        kvh.level_info(4)
+    assert e.value.status == 2
+    assert kvh.status_string(6) == "page id outside the pool"
+
+
+def test_level_bytes_matches_oracle(kvh):
+    for l in (1, 3, 32, 80):
+        for c in (32, 96, 128, 1024, 4096):
+            for n in (1, 2, 15, 16, 17, 31, 32, 33, 64, 100, 255, 256):
+                for k in range(4):
+                    assert kvh.level_bytes(k, l, c, n) == oracle.level_bytes(k, l, c, n) > 0
+
+
+@pytest.mark.parametrize("args,status", [
+    ((4, 1, 32, 1), 2), ((-1, 1, 32, 1), 2), ((0, 0, 32, 1), 3), ((0, 1, 48, 1), 3),
+    ((0, 1, 32, 0), 3), ((0, 1, 32, 257), 3),
+])
+def test_level_bytes_rejects(kvh, args, status):
+    with pytest.raises(kvh.KvhError) as e:
+        kvh.level_bytes(*args)
+    assert e.value.status == status
+    assert oracle.level_bytes(*args) == 0
+
+
+def test_plan_chunks_matches_oracle(kvh):
+    l, c = 4, 64
+    for N, levels in [(256, 2), (1000, [0, 1, 2, 3]), (257, [3, 0]), (5, 1), (8192, 3)]:
+        descs, total = kvh.plan_chunks(l, c, N, levels, stream_base=256, pt_base=7)
+        ntoks, lv, offsets = oracle.chunk_plan(N, levels, l, c)
+        assert total == offsets[-1]
+        assert descs["stream_off"].tolist() == [256 + o for o in offsets[:-1]]
+        assert descs["n_tok"].tolist() == ntoks and descs["level"].tolist() == lv
+        assert descs["pt_off"].tolist() == [7 + 16 * i for i in range(len(ntoks))]
+        assert not descs["reserved"].any()
+    descs, _ = kvh.plan_chunks(l, c, 600, 0, page_tokens=32)
+    assert descs["pt_off"].tolist() == [0, 8, 16]
+
+
+def test_plan_chunks_rejects(kvh):
+    for kwargs, status in [(dict(stream_base=64), 4), (dict(page_tokens=24), 3), (dict(pt_base=-1), 1)]:
+        with pytest.raises(kvh.KvhError) as e:
+            kvh.plan_chunks(2, 64, 300, 1, **kwargs)
+        assert e.value.status == status
+    with pytest.raises(kvh.KvhError) as e:
+        kvh.plan_chunks(2, 64, 300, [1, 9])
+    assert e.value.status == 2
+    with pytest.raises(ValueError):
+        kvh.plan_chunks(2, 64, 300, [1])
+
+
+def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(kvh):
+    L = kvh.lib()
+    buf = (ctypes.c_uint8 * 4096)()
+    a = (ctypes.addressof(buf) + 127) & ~127          # host memory: never dereferenced on these paths
+    assert L.kvh_encode(None, 1, 256, 32, 0, a, 1 << 20, None, None) == 1
+    assert L.kvh_encode(a, 1, 0, 32, 0, a, 1 << 20, None, None) == 1
+    assert L.kvh_encode(a, 1, 256, 32, 7, a, 1 << 20, None, None) == 2
+    assert L.kvh_encode(a, 1, 256, 40, 0, a, 1 << 20, None, None) == 3
+    assert L.kvh_encode(a + 8, 1, 256, 32, 0, a, 1 << 20, None, None) == 4
+    assert L.kvh_encode(a, 1, 256, 32, 0, a + 64, 1 << 20, None, None) == 4
+    assert L.kvh_encode(a, 1, 256, 32, 0, a, 100, None, None) == 5
+    assert L.kvh_encode_chunks(a, 1, 600, 32, a, 2, a, 1 << 20, None, None) == 3      # 600 tokens = 3 chunks
+    pool = kvh.binding._PoolStruct(a, 2 * 8 * 16 * 32, 8 * 16 * 32, 16 * 32, 8, 16, 1, 32)
+    assert L.kvh_decode_to_pages(None, 0, 16, a, ctypes.byref(pool), None, None) == 1
+    assert L.kvh_decode_to_pages(a, 4, 16, a, ctypes.byref(pool), None, None) == 2
+    assert L.kvh_decode_to_pages(a, 0, 300, a, ctypes.byref(pool), None, None) == 3
+    assert L.kvh_decode_to_pages(a + 16, 0, 16, a, ctypes.byref(pool), None, None) == 4
+    bad = kvh.binding._PoolStruct(a, 2 * 8 * 16 * 32, 8 * 16 * 32, 16 * 32 + 4, 8, 16, 1, 32)
+    assert L.kvh_decode_to_pages(a, 0, 16, a, ctypes.byref(bad), None, None) == 4
+    bad = kvh.binding._PoolStruct(a, 2 * 8 * 16 * 32, 8 * 16 * 32, 16 * 32, 8, 24, 1, 32)
+    assert L.kvh_decode_to_pages(a, 0, 16, a, ctypes.byref(bad), None, None) == 3
+    assert L.kvh_decode_batch(a, 4096, None, 1, a, 16, ctypes.byref(pool), None, None) == 1
+    assert L.kvh_decode_batch(a, 4096, a, 0, a, 16, ctypes.byref(pool), None, None) == 0   # nothing to do
+
+
+def test_missing_library_fails_loudly(kvh, monkeypatch, tmp_path):
+    from paper_2509_00105_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "libkvh.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.lib()
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2509_00105_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f
