@@ -5,7 +5,11 @@
 #include <stdint.h>
 
 #include "kvh.h"
+#include <stdlib.h>
+#include <string.h>
+
 #include "kvh_decode.cuh"
+#include "kvh_decode_tma.cuh"
 #include "kvh_encode.cuh"
 #include "kvh_format.cuh"
 
@@ -54,10 +58,34 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     p.page_stride = pool->page_stride;
     p.num_pages = pool->num_pages;
     p.page_tokens = pool->page_tokens;
+    p.page_shift = 0;
+    while ((1 << p.page_shift) < pool->page_tokens) ++p.page_shift;   // divisors of 256 are powers of two
     p.l = pool->n_layers;
     p.c = pool->n_channels;
     const unsigned grid = grid_for(n_chunks, p.l);
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    // KVH_DECODE_PATH=direct forces the one-CTA-per-tile kernel (a measurement aid); the
+    // persistent TMA kernel needs a tile to fit a shared-memory stage and at most 2 pages per tile.
+    const char *force = getenv("KVH_DECODE_PATH");
+    const bool want_tma = !(force && strcmp(force, "direct") == 0);
+    if (want_tma && p.c <= kTmaMaxChannels && p.page_tokens >= 16) {
+        int dev = 0, sms = 0, per_sm = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return KVH_ERR_CUDA;
+        const uint32_t stage = tma_stage_bytes(p.c);
+        int stages = (int)((112u * 1024u) / stage);           // two CTAs per SM when c = 1024
+        stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
+        const size_t dyn = (size_t)stages * stage;
+        if (cudaFuncSetAttribute(decode_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_tma_kernel, kTmaThreads, dyn) != cudaSuccess ||
+            per_sm < 1)
+            return KVH_ERR_CUDA;
+        const int64_t resident = (int64_t)sms * per_sm;
+        const unsigned pgrid = (unsigned)(grid < resident ? grid : resident);
+        decode_tma_kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages);
+        return launch_status();
+    }
     decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
     return launch_status();
 }

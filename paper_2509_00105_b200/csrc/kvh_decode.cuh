@@ -25,7 +25,7 @@ struct DecodeParams {
     int64_t page_table_len;
     uint16_t *pool;
     int64_t layer_stride, kv_stride, page_stride;
-    int32_t num_pages, page_tokens, l, c;
+    int32_t num_pages, page_tokens, page_shift, l, c;   // page_tokens == 1 << page_shift
     int32_t *status;
 };
 
@@ -71,15 +71,13 @@ __device__ __forceinline__ uint64_t load_codes8(const uint8_t *codes, uint64_t e
 }
 
 // Destination row of chunk token T for this plane, or nullptr if its page id is out of range.
-__device__ __forceinline__ uint16_t *page_row(const DecodeParams &p, const int32_t *page_ids,
-                                              uint16_t *plane, int T)
+__device__ __forceinline__ uint16_t *page_row(const DecodeParams &p, int32_t pg, uint16_t *plane, int T)
 {
-    const int32_t pg = __ldg(page_ids + T / p.page_tokens);
     if ((uint32_t)pg >= (uint32_t)p.num_pages) {
         report(p.status, KVH_ERR_PAGE_OOB);
         return nullptr;
     }
-    return plane + (int64_t)pg * p.page_stride + (int64_t)(T % p.page_tokens) * p.c;
+    return plane + (int64_t)pg * p.page_stride + (int64_t)(T & (p.page_tokens - 1)) * p.c;
 }
 
 template <int BITS>
@@ -89,13 +87,15 @@ __device__ __forceinline__ void decode_tile(const DecodeParams &p, const uint8_t
 {
     const int c = p.c;
     const int V8 = c >> 3;                               // 8-channel vectors per token row
-    const int cstep = V8 <= kThreads ? V8 : kThreads;
+    const int cstep = V8 <= kThreads ? V8 : kThreads;     // a multiple of 4: V8 is, and so is kThreads
     const int rpp = V8 <= kThreads ? kThreads / V8 : 1;   // token rows the CTA covers per pass
     const int my_row = threadIdx.x / cstep;
     const int my_cv = threadIdx.x - my_row * cstep;
-    if (my_row >= rpp) return;
+    if (my_row >= rpp) return;                           // whole quads of lanes leave together
     const int t0 = tile * kTileTokens;
-    constexpr int U = 4;                                 // rows in flight per thread
+    constexpr int U = 8;                                 // rows in flight per thread
+    const int lane = threadIdx.x & 31;
+    const uint32_t quad = 0xfu << (lane & ~3);           // the 4 lanes that share a V group
 
     for (int cv = my_cv; cv < V8; cv += cstep) {
         float lo[8], sc[8];
@@ -112,11 +112,13 @@ __device__ __forceinline__ void decode_tile(const DecodeParams &p, const uint8_t
             uint4 raw[U];
             uint64_t cd[U];
             uint32_t vm[U];
+            int32_t pg[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int t = tb + u * rpp;
                 if (t < nt) {
                     const uint64_t e = (uint64_t)(t0 + t) * c + 8 * cv;
+                    pg[u] = __ldg(page_ids + ((t0 + t) >> p.page_shift));
                     if constexpr (BITS == 16) {
                         raw[u] = __ldcs(reinterpret_cast<const uint4 *>(codes + 2 * e));
                     } else {
@@ -127,26 +129,44 @@ __device__ __forceinline__ void decode_tile(const DecodeParams &p, const uint8_t
                     }
                 }
             }
+            // V: the 4 lanes of a quad share each row's group; each derives the scale of every
+            // fourth row and hands it round, so a row costs a quarter of a division per lane
+            float vsc[U / 4];
+            if constexpr (BITS < 16) {
+                if (kv == 1) {
+#pragma unroll
+                    for (int j = 0; j < U / 4; ++j) {
+                        const int u = 4 * j + (lane & 3);
+                        float l1;
+                        vsc[j] = 0.0f;
+                        if (tb + u * rpp < nt) {
+                            uint32_t m = vm[4 * j];
+                            if ((lane & 3) == 1) m = vm[4 * j + 1];
+                            if ((lane & 3) == 2) m = vm[4 * j + 2];
+                            if ((lane & 3) == 3) m = vm[4 * j + 3];
+                            decode_params<BITS>(m, l1, vsc[j]);
+                        }
+                    }
+                }
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int t = tb + u * rpp;
-                if (t < nt) {
-                    uint16_t *row = page_row(p, page_ids, plane, t0 + t);
-                    if (row) {
-                        uint4 v;
-                        if constexpr (BITS == 16) {
-                            v = raw[u];
-                        } else {
-                            if (kv == 1) {
-                                float l1, s1;
-                                decode_params<BITS>(vm[u], l1, s1);
+                if (t < nt) {                                // uniform within a quad
+                    uint4 v;
+                    if constexpr (BITS == 16) {
+                        v = raw[u];
+                    } else {
+                        if (kv == 1) {
+                            const float s1 = __shfl_sync(quad, vsc[u >> 2], (lane & ~3) | (u & 3));
+                            const float l1 = bf16_lo_to_f32(vm[u]);
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) { lo[i] = l1; sc[i] = s1; }
-                            }
-                            v = dequant8<BITS>(cd[u], lo, sc);
+                            for (int i = 0; i < 8; ++i) { lo[i] = l1; sc[i] = s1; }
                         }
-                        *reinterpret_cast<uint4 *>(row + 8 * cv) = v;
+                        v = dequant8<BITS>(cd[u], lo, sc);
                     }
+                    uint16_t *row = page_row(p, pg[u], plane, t0 + t);
+                    if (row) *reinterpret_cast<uint4 *>(row + 8 * cv) = v;
                 }
             }
         }
@@ -163,7 +183,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const DecodeParams p)
 
     const kvh_chunk_desc d = p.descs ? p.descs[chunk] : p.single;
     int err = check_desc(d, p.l, p.c, p.streams_bytes);
-    const int npages = (d.n_tok + p.page_tokens - 1) / p.page_tokens;
+    const int npages = (d.n_tok + p.page_tokens - 1) >> p.page_shift;
     if (err == KVH_OK && (d.pt_off < 0 || (int64_t)d.pt_off + npages > p.page_table_len))
         err = KVH_ERR_BUFFER_TOO_SMALL;
     if (err != KVH_OK) {

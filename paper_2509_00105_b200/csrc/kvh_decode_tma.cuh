@@ -1,0 +1,408 @@
+// Persistent, TMA-fed decode kernel (the fast path for c <= 1024, pages of >= 16 tokens).
+//
+// One CTA (or a few) per SM loops over work units.  A producer warp walks the CTA's share of
+// (chunk, layer, K|V, 32-token tile) tiles, resolves descriptors and page ids, and streams each
+// unit's codes and group metadata from HBM into a ring of shared-memory stages with 1-D bulk
+// async copies (cp.async.bulk, completion counted on an mbarrier).  Eight consumer warps unpack,
+// dequantise and write full 16-byte vectors of page rows.  Copies for the next stages are always
+// in flight while the current one is being expanded, so HBM latency is off the critical path and
+// the kernel runs at the speed of its writes (2 of the (b+1)/8 + 2 bytes moved per element).
+//
+// A unit is a 32-token tile of a quantised plane (<= 32*c bytes of codes + 4*c bytes of metadata)
+// or one 16-token half of a raw bf16 tile (32*c bytes), so every unit fits one stage.
+//
+// Every wait is bounded: a wait that runs out reports KVH_ERR_TIMEOUT, raises the CTA's abort
+// flag and the CTA leaves after its copies in flight have landed.
+#pragma once
+
+#include "kvh_decode.cuh"
+#include "kvh_format.cuh"
+
+namespace kvh {
+
+constexpr int kConsumerThreads = 256;
+constexpr int kTmaThreads = kConsumerThreads + 32;      // + one producer warp
+constexpr int kMaxStages = 8;
+constexpr int kTmaMaxChannels = 1024;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct UnitInfo {
+    int32_t bits;        // 16, 8, 4, 2; 0 marks the end of the CTA's work
+    int32_t kv;          // 0 K, 1 V
+    int32_t row0;        // first token of the unit within its chunk
+    int32_t nrows;       // tokens in the unit (1..32)
+    int32_t pg0, pg1;    // page ids of the page holding row0 and of the next one
+    uint16_t *plane;     // pool + layer*layer_stride + kv*kv_stride
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a phase of an mbarrier; false if the time limit ran out or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long start = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag || global_ns() - start > kWaitLimitNs) return false;
+    }
+}
+// 1-D bulk copy global -> this CTA's shared memory; bytes is a multiple of 16, both ends 16-byte aligned.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+__host__ __device__ __forceinline__ uint32_t tma_stage_bytes(int c) { return (36u * (uint32_t)c + 127u) & ~127u; }
+__host__ __device__ __forceinline__ uint32_t round16(uint32_t x) { return (x + 15u) & ~15u; }
+
+// ---- dequantisation of 8 consecutive codes with few instructions per element ----------------
+//
+// A code is never shifted down to bit 0.  For 2- and 4-bit codes the field is masked in place and
+// OR-ed into the mantissa of 2^23 (one logic op), so subtracting 2^23 leaves q * 2^pos exactly;
+// the group's scale is pre-multiplied by 2^-pos (exact: a power of two, and scales are >= 2^-108
+// or zero), hence fma(q * 2^pos, scale * 2^-pos, lo) has the same exact product, the same single
+// rounding and the same result as fma(q, scale, lo).  8-bit codes are placed by a byte permute.
+template <int BITS> struct Pos;
+template <> struct Pos<2> {      // fields of the low byte of a 16-bit half: bits 0, 2, 4, 6
+    static constexpr int kFieldsPerWord = 4;
+    __device__ static __forceinline__ float prescale(int i) { return 1.0f / (float)(1 << (2 * (i & 3))); }
+};
+template <> struct Pos<4> {      // fields of a 16-bit half: bits 0, 4, 8, 12
+    static constexpr int kFieldsPerWord = 4;
+    __device__ static __forceinline__ float prescale(int i) { return 1.0f / (float)(1 << (4 * (i & 3))); }
+};
+template <> struct Pos<8> {
+    static constexpr int kFieldsPerWord = 4;
+    __device__ static __forceinline__ float prescale(int) { return 1.0f; }
+};
+
+// q_i * 2^pos(i) as a float, for i = 0..7, from the 8 codes of one thread
+template <int BITS>
+__device__ __forceinline__ void spread8(const uint8_t *src, float (&x)[8])
+{
+    constexpr uint32_t magic = 0x4b000000u;
+    uint32_t m[8];
+    if constexpr (BITS == 2) {
+        const uint32_t w = *reinterpret_cast<const uint16_t *>(src);
+        const uint32_t t = w >> 8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            m[i] = (w & (3u << (2 * i))) | magic;
+            m[i + 4] = (t & (3u << (2 * i))) | magic;
+        }
+    } else if constexpr (BITS == 4) {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(src);
+        const uint32_t t = w >> 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            m[i] = (w & (15u << (4 * i))) | magic;
+            m[i + 4] = (t & (15u << (4 * i))) | magic;
+        }
+    } else {
+        const uint2 w = *reinterpret_cast<const uint2 *>(src);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            m[i] = __byte_perm(w.x, magic, 0x7440 + i);       // bytes: code, 0, 0, 0x4b
+            m[i + 4] = __byte_perm(w.y, magic, 0x7440 + i);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = __fsub_rn(__uint_as_float(m[i]), 8388608.0f);
+}
+
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    return make_uint4(pack_bf16x2_rn(f[0], f[1]), pack_bf16x2_rn(f[2], f[3]),
+                      pack_bf16x2_rn(f[4], f[5]), pack_bf16x2_rn(f[6], f[7]));
+}
+
+// Rows of a unit are dealt to threads in runs of `rpt` consecutive rows (a power of two, so a run
+// never straddles a page); `cv` is the thread's 8-channel vector within the row.
+struct RowRun {
+    int cv, first, count;       // count == 0 for idle threads
+    uint16_t *dst;              // first row's destination (already offset by cv), nullptr if none
+};
+
+__device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u)
+{
+    const int V8 = p.c >> 3;                              // <= 128
+    const int rpp = kConsumerThreads / V8;                // row groups the CTA holds, >= 2
+    int rpt = 1;
+    while (rpt * rpp < kTileTokens) rpt <<= 1;            // rows per thread: 16 when c = 1024
+    const int g = threadIdx.x / V8;
+    RowRun r;
+    r.cv = threadIdx.x - g * V8;
+    r.first = g * rpt;
+    r.count = g < rpp ? max(0, min(rpt, u.nrows - r.first)) : 0;
+    r.dst = nullptr;
+    if (r.count > 0) {
+        const int T = u.row0 + r.first;
+        const int32_t pg = (T >> p.page_shift) == (u.row0 >> p.page_shift) ? u.pg0 : u.pg1;
+        r.dst = page_row(p, pg, u.plane, T);              // reports an out-of-range page id
+        if (r.dst) r.dst += 8 * r.cv; else r.count = 0;
+    }
+    return r;
+}
+
+__device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
+{
+    const RowRun r = row_run(p, u);
+    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * p.c + 8 * r.cv));
+    uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
+    const int stride = p.c >> 3;                          // uint4 per row
+#pragma unroll 4
+    for (int k = 0; k < r.count; ++k) dst[(size_t)k * stride] = src[(size_t)k * stride];
+}
+
+template <int BITS>
+__device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
+                                          const uint8_t *meta)
+{
+    const RowRun r = row_run(p, u);
+    if (r.count == 0) return;
+    float lo[8], sc[8];
+    {
+        const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * r.cv;
+        const uint4 m0 = m[0], m1 = m[1];
+        const uint32_t w[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            decode_params<BITS>(w[i], lo[i], sc[i]);
+            sc[i] = __fmul_rn(sc[i], Pos<BITS>::prescale(i));
+        }
+    }
+    const uint32_t row_bytes = (uint32_t)p.c * BITS / 8;
+    const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
+    uint16_t *dst = r.dst;
+#pragma unroll 2
+    for (int k = 0; k < r.count; ++k) {
+        float x[8], f[8];
+        spread8<BITS>(src, x);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], sc[i], lo[i]);
+        *reinterpret_cast<uint4 *>(dst) = pack8(f);
+        src += row_bytes;
+        dst += p.c;
+    }
+}
+
+template <int BITS>
+__device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
+                                          const uint8_t *meta)
+{
+    const RowRun r = row_run(p, u);
+    const int lane = threadIdx.x & 31;
+    const uint32_t quad = 0xfu << (lane & ~3);            // the 4 lanes that share every V group
+    const int groups = p.c / kGroup;
+    const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)r.first * groups + (r.cv >> 2);
+    const uint32_t row_bytes = (uint32_t)p.c * BITS / 8;
+    const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
+    uint16_t *dst = r.dst;
+    // r.count is the same for the 4 lanes of a quad (they share the row group), so the shuffles
+    // below are executed by whole quads
+    for (int kb = 0; kb < r.count; kb += 4) {
+        // each lane of the quad derives the scale of one of the next 4 rows: a quarter of a
+        // division per row and lane
+        float mine = 0.0f, unused;
+        const int kq = kb + (lane & 3);
+        if (kq < r.count) decode_params<BITS>(mrow[(size_t)kq * groups], unused, mine);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (kb + j < r.count) {
+                const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
+                const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
+                float s[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[i] = __fmul_rn(s0, Pos<BITS>::prescale(i));
+                float x[8], f[8];
+                spread8<BITS>(src, x);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], s[i & 3], l1);
+                *reinterpret_cast<uint4 *>(dst) = pack8(f);
+                src += row_bytes;
+                dst += p.c;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodeParams p, const int n_chunks,
+                                                                 const int n_stages)
+{
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ UnitInfo info[kMaxStages];
+    __shared__ int abort_flag;
+
+    const uint32_t stage_bytes = tma_stage_bytes(p.c);
+    const uint32_t meta_off = 32u * p.c;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerThreads / 32);
+        }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerThreads / 32) {
+        // ------------------------------ producer warp ------------------------------
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        int cur_chunk = -1;
+        bool valid = false;
+        kvh_chunk_desc d = p.single;
+        int32_t my_pg = 0;                           // lane j holds page id j of the current chunk
+        LayerLayout L = layer_layout(0, p.c, 1);
+        uint32_t unit = 0;
+        bool ok = true;
+
+        auto emit = [&](int bits, int kv, int row0, int nrows, uint16_t *plane, const uint8_t *codes_src,
+                        uint32_t codes_bytes, const uint8_t *meta_src, uint32_t meta_bytes) -> bool {
+            const int s = unit % n_stages;
+            if (unit >= (uint32_t)n_stages) {
+                bool w = true;
+                if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / n_stages) - 1) & 1, &abort_flag);
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w) return false;
+            }
+            const int pidx = row0 >> p.page_shift;
+            const int32_t pg0 = __shfl_sync(0xffffffffu, my_pg, pidx & 31);
+            const int32_t pg1 = __shfl_sync(0xffffffffu, my_pg, (pidx + 1) & 31);
+            if (lane == 0) {
+                UnitInfo &u = info[s];
+                u.bits = bits; u.kv = kv; u.row0 = row0; u.nrows = nrows; u.pg0 = pg0; u.pg1 = pg1; u.plane = plane;
+                uint8_t *st = stage_mem + (size_t)s * stage_bytes;
+                if (bits == 0) {
+                    mbar_arrive(&full_bar[s]);
+                } else {
+                    mbar_arrive_expect_tx(&full_bar[s], codes_bytes + meta_bytes);
+                    bulk_load(st, codes_src, codes_bytes, &full_bar[s]);
+                    if (meta_bytes) bulk_load(st + meta_off, meta_src, meta_bytes, &full_bar[s]);
+                }
+            }
+            ++unit;
+            return true;
+        };
+
+        for (int64_t tile_id = blockIdx.x; ok && tile_id < total_tiles; tile_id += gridDim.x) {
+            const int tile = (int)(tile_id % kTilesPerChunk);
+            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int kv = (int)(plane_id & 1);
+            const int layer = (int)((plane_id >> 1) % p.l);
+            const int chunk = (int)((plane_id >> 1) / p.l);
+            if (chunk != cur_chunk) {
+                cur_chunk = chunk;
+                if (p.descs) d = p.descs[chunk];
+                int err = check_desc(d, p.l, p.c, p.streams_bytes);
+                const int npages = (d.n_tok + p.page_tokens - 1) >> p.page_shift;
+                if (err == KVH_OK && (d.pt_off < 0 || (int64_t)d.pt_off + npages > p.page_table_len))
+                    err = KVH_ERR_BUFFER_TOO_SMALL;
+                valid = err == KVH_OK;
+                if (!valid) {
+                    if (lane == 0) report(p.status, err);
+                } else {
+                    my_pg = lane < npages ? __ldg(p.page_table + d.pt_off + lane) : 0;
+                    L = layer_layout(d.level, p.c, d.n_tok);
+                }
+            }
+            if (!valid) continue;
+            const int t0 = tile * kTileTokens;
+            const int nt = min(kTileTokens, d.n_tok - t0);
+            if (nt <= 0) continue;
+            const uint8_t *lay = p.streams + d.stream_off + (uint64_t)layer * L.layer_bytes();
+            const uint8_t *meta = lay + L.meta_off(kv);
+            const uint8_t *codes = lay + L.codes_off(kv);
+            uint16_t *plane = p.pool + (int64_t)layer * p.layer_stride + (int64_t)kv * p.kv_stride;
+            if (d.level == 0) {
+                for (int h = 0; ok && h < nt; h += 16) {
+                    const int rows = min(16, nt - h);
+                    ok = emit(16, kv, t0 + h, rows, plane, codes + 2 * (uint64_t)(t0 + h) * p.c,
+                              round16(2u * rows * p.c), nullptr, 0);
+                }
+            } else {
+                const int b = level_bits(d.level);
+                const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
+                const uint8_t *msrc = kv == 0 ? meta + 4 * (uint64_t)tile * p.c
+                                              : meta + 4 * (uint64_t)t0 * (p.c / kGroup);
+                const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * (p.c / kGroup));
+                ok = emit(b, kv, t0, nt, plane, codes + (uint64_t)t0 * p.c * b / 8, cbytes, msrc, mbytes);
+            }
+        }
+        if (ok) ok = emit(0, 0, 0, 0, nullptr, nullptr, 0, nullptr, 0);       // end marker
+        if (!ok && lane == 0) {
+            report(p.status, KVH_ERR_TIMEOUT);
+            abort_flag = 1;
+        }
+        // Leave only after every copy issued has landed: a normal run has seen them all consumed;
+        // after an abort the last n_stages units may still be in flight.
+        if (lane == 0) {
+            int never = 0;                           // the drain ignores the abort flag
+            const uint32_t first = unit > (uint32_t)n_stages ? unit - n_stages : 0;
+            for (uint32_t w = first; w < unit; ++w)
+                (void)mbar_wait(&full_bar[w % n_stages], (w / n_stages) & 1, &never);
+        }
+    } else {
+        // ------------------------------ consumer warps ------------------------------
+        for (uint32_t unit = 0;; ++unit) {
+            const int s = unit % n_stages;
+            if (!mbar_wait(&full_bar[s], (unit / n_stages) & 1, &abort_flag)) {
+                report(p.status, KVH_ERR_TIMEOUT);
+                abort_flag = 1;
+                break;
+            }
+            const UnitInfo u = info[s];
+            if (u.bits == 0) break;
+            const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
+            const uint8_t *mt = st + meta_off;
+            switch (u.bits * 2 + u.kv) {                      // uniform per CTA
+            case 32: case 33: consume_raw(p, u, st); break;
+            case 16: consume_k<8>(p, u, st, mt); break;
+            case 17: consume_v<8>(p, u, st, mt); break;
+            case 8: consume_k<4>(p, u, st, mt); break;
+            case 9: consume_v<4>(p, u, st, mt); break;
+            case 4: consume_k<2>(p, u, st, mt); break;
+            default: consume_v<2>(p, u, st, mt); break;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[s]);
+        }
+    }
+}
+
+}  // namespace kvh

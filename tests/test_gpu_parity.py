@@ -77,9 +77,16 @@ SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("path", ["default", "direct"])
 @pytest.mark.parametrize("l,c,N", SHAPES)
 @pytest.mark.parametrize("level", [0, 1, 2, 3])
-def test_encode_and_decode_match_oracle(kvh, l, c, N, level):
+def test_encode_and_decode_match_oracle(kvh, monkeypatch, l, c, N, level, path):
+    # "default" takes the persistent TMA decode kernel where it applies (c <= 1024); "direct"
+    # forces the one-CTA-per-tile kernel on every shape
+    if path == "direct":
+        monkeypatch.setenv("KVH_DECODE_PATH", "direct")
+    else:
+        monkeypatch.delenv("KVH_DECODE_PATH", raising=False)
     kv = workloads.make_kv(l, N, c, seed=1000 * level + N + c, device="cuda")
     kv_np = to_np16(kv).copy()
     special_values(kv_np, N)
