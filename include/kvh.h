@@ -153,6 +153,35 @@ kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes,
                             const int32_t *page_table, int64_t page_table_len,
                             const kvh_pool *pool, int32_t *dev_status, void *stream);
 
+/* ---- host-tier entry points: the stored form lives in (pinned) host memory ------------------
+ *
+ * The paper keeps compressed entries in DRAM and SSD and loads them on a hit; its loading delay
+ * is size / bandwidth (utility definition).  These two calls move a context between pinned host
+ * memory and the GPU in slices of about slice_bytes, overlapping the PCIe copy of one slice (on
+ * copy_stream) with the kernel of the previous one (on stream).  descs_host [host] and descs_dev
+ * [device] hold the same n_chunks descriptors, laid out by kvh_plan_chunks with ascending,
+ * contiguous stream offsets; offsets index both the host buffer and dev_staging [device,
+ * 128-byte aligned, staging_bytes long].  If host_status [host, pinned] is not NULL, *dev_status
+ * is copied to it on `stream` after the last kernel.  copy_stream must be a non-NULL stream
+ * other than `stream`, created non-blocking if `stream` is the default stream; the calls return
+ * without waiting and create no device memory. */
+
+/* Cache hit on the host tier: copy the stored chunks host -> device and decode them into the
+ * pool.  The load path of the paper's hierarchy. */
+kvh_status kvh_load_host(const void *host_streams, void *dev_staging, uint64_t staging_bytes,
+                         const kvh_chunk_desc *descs_host, const kvh_chunk_desc *descs_dev,
+                         int n_chunks, const int32_t *page_table, int64_t page_table_len,
+                         const kvh_pool *pool, int32_t *dev_status, int32_t *host_status,
+                         uint64_t slice_bytes, void *copy_stream, void *stream);
+
+/* Store to the host tier: encode the context kv [device] chunk by chunk and copy the streams
+ * device -> host.  descs describe the whole context (chunk i = tokens [256 i, ...)). */
+kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                          const kvh_chunk_desc *descs_host, const kvh_chunk_desc *descs_dev,
+                          int n_chunks, void *dev_staging, uint64_t staging_bytes, void *host_out,
+                          int32_t *dev_status, int32_t *host_status, uint64_t slice_bytes,
+                          void *copy_stream, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

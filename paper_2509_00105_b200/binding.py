@@ -73,6 +73,11 @@ def lib() -> ctypes.CDLL:
         L.kvh_decode_to_pages.argtypes = [vp, i32, i32, vp, ctypes.POINTER(_PoolStruct), vp, vp]
         L.kvh_decode_batch.restype = i32
         L.kvh_decode_batch.argtypes = [vp, u64, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp]
+        L.kvh_load_host.restype = i32
+        L.kvh_load_host.argtypes = [vp, vp, u64, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp,
+                                    u64, vp, vp]
+        L.kvh_store_host.restype = i32
+        L.kvh_store_host.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, u64, vp, vp, vp, u64, vp, vp]
         _lib = L
     return _lib
 
@@ -206,3 +211,37 @@ def decode_batch(streams: torch.Tensor, descs_dev: torch.Tensor, n_chunks: int, 
     _check(lib().kvh_decode_batch(streams.data_ptr(), streams.numel(), descs_dev.data_ptr(), n_chunks,
                                   page_table.data_ptr(), page_table.numel(), ctypes.byref(pool.struct),
                                   _ptr(dev_status), _stream()), "kvh_decode_batch")
+
+
+def load_host(host_streams: torch.Tensor, staging: torch.Tensor, descs: np.ndarray, descs_dev: torch.Tensor,
+              page_table: torch.Tensor, pool: Pool, dev_status: torch.Tensor | None,
+              host_status: torch.Tensor | None, copy_stream: torch.cuda.Stream, slice_bytes: int = 0) -> None:
+    """Host-tier cache hit: copy the stored chunks from pinned host memory and decode them into the
+    pool, slice by slice, the copy on copy_stream overlapping the decode on the current stream."""
+    assert host_streams.is_pinned() and host_streams.dtype == torch.uint8 and descs.dtype == DESC_DTYPE
+    assert staging.is_cuda and staging.dtype == torch.uint8
+    assert host_status is None or (host_status.is_pinned() and host_status.dtype == torch.int32)
+    need = int(descs["stream_off"][-1]) + level_bytes(int(descs["level"][-1]), pool.struct.n_layers,
+                                                       pool.struct.n_channels, int(descs["n_tok"][-1]))
+    if host_streams.numel() < need:
+        raise KvhError(5, "load_host")
+    _check(lib().kvh_load_host(host_streams.data_ptr(), staging.data_ptr(), staging.numel(), descs.ctypes.data,
+                               descs_dev.data_ptr(), len(descs), page_table.data_ptr(), page_table.numel(),
+                               ctypes.byref(pool.struct), _ptr(dev_status), _ptr(host_status), slice_bytes,
+                               copy_stream.cuda_stream, _stream()), "kvh_load_host")
+
+
+def store_host(kv: torch.Tensor, descs: np.ndarray, descs_dev: torch.Tensor, staging: torch.Tensor,
+               host_out: torch.Tensor, dev_status: torch.Tensor | None, host_status: torch.Tensor | None,
+               copy_stream: torch.cuda.Stream, slice_bytes: int = 0) -> None:
+    """Store to the host tier: encode the context slice by slice on the current stream and copy
+    each slice's streams to pinned host memory on copy_stream."""
+    l, N, c = _check_kv(kv)
+    assert host_out.is_pinned() and host_out.dtype == torch.uint8 and descs.dtype == DESC_DTYPE
+    need = int(descs["stream_off"][-1]) + level_bytes(int(descs["level"][-1]), l, c, int(descs["n_tok"][-1]))
+    if host_out.numel() < need:
+        raise KvhError(5, "store_host")
+    _check(lib().kvh_store_host(kv.data_ptr(), l, N, c, descs.ctypes.data, descs_dev.data_ptr(), len(descs),
+                                staging.data_ptr(), staging.numel(), host_out.data_ptr(), _ptr(dev_status),
+                                _ptr(host_status), slice_bytes, copy_stream.cuda_stream, _stream()),
+           "kvh_store_host")

@@ -255,4 +255,135 @@ kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes, co
     return launch_decode(p, pool, n_chunks, stream);
 }
 
+// ---- host tier ------------------------------------------------------------------------------
+
+namespace {
+
+// Descriptors must tile [first offset, end) without gaps, in order, so a slice of chunks is one
+// contiguous byte range on both sides of the PCIe copy.
+kvh_status check_contiguous(const kvh_chunk_desc *d, int n, int l, int c, uint64_t capacity)
+{
+    uint64_t expect = d[0].stream_off;
+    for (int i = 0; i < n; ++i) {
+        if (d[i].level < 0 || d[i].level >= kNumLevels) return KVH_ERR_BAD_LEVEL;
+        if (d[i].n_tok < 1 || d[i].n_tok > kChunkTokens) return KVH_ERR_BAD_SHAPE;
+        if (d[i].stream_off % KVH_SECTION_ALIGN) return KVH_ERR_MISALIGNED;
+        if (d[i].stream_off != expect) return KVH_ERR_INVALID_ARG;
+        expect += chunk_bytes(d[i].level, l, c, d[i].n_tok);
+    }
+    return expect <= capacity ? KVH_OK : KVH_ERR_BUFFER_TOO_SMALL;
+}
+
+struct Slice { int first, count; uint64_t off, bytes; };
+
+// Next slice of chunks starting at `first`: at least one chunk, about slice_bytes long.
+Slice next_slice(const kvh_chunk_desc *d, int n, int first, int l, int c, uint64_t slice_bytes)
+{
+    Slice s{first, 0, d[first].stream_off, 0};
+    while (first + s.count < n && (s.count == 0 || s.bytes < slice_bytes)) {
+        s.bytes += chunk_bytes(d[first + s.count].level, l, c, d[first + s.count].n_tok);
+        ++s.count;
+    }
+    return s;
+}
+
+// Make `waiter` wait for everything enqueued on `signaller` so far.
+bool chain(cudaStream_t signaller, cudaStream_t waiter)
+{
+    cudaEvent_t ev;
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return false;
+    const bool ok = cudaEventRecord(ev, signaller) == cudaSuccess &&
+                    cudaStreamWaitEvent(waiter, ev, 0) == cudaSuccess;
+    cudaEventDestroy(ev);            // released once the recorded work completes
+    return ok;
+}
+
+}  // namespace
+
+kvh_status kvh_load_host(const void *host_streams, void *dev_staging, uint64_t staging_bytes,
+                         const kvh_chunk_desc *descs_host, const kvh_chunk_desc *descs_dev, int n_chunks,
+                         const int32_t *page_table, int64_t page_table_len, const kvh_pool *pool,
+                         int32_t *dev_status, int32_t *host_status, uint64_t slice_bytes,
+                         void *copy_stream, void *stream)
+{
+    if (!host_streams || !dev_staging || !descs_host || !descs_dev || !page_table || n_chunks <= 0 ||
+        page_table_len < 0 || !copy_stream || copy_stream == stream || (host_status && !dev_status))
+        return KVH_ERR_INVALID_ARG;
+    const kvh_status ps = check_pool(pool);
+    if (ps != KVH_OK) return ps;
+    if (!aligned(dev_staging, KVH_SECTION_ALIGN) || !aligned(descs_dev, 8) || !aligned(page_table, 4))
+        return KVH_ERR_MISALIGNED;
+    const kvh_status cs = check_contiguous(descs_host, n_chunks, pool->n_layers, pool->n_channels, staging_bytes);
+    if (cs != KVH_OK) return cs;
+    if (slice_bytes == 0) slice_bytes = 64ull << 20;
+    cudaStream_t cp = static_cast<cudaStream_t>(copy_stream), st = static_cast<cudaStream_t>(stream);
+    if (!chain(st, cp)) return KVH_ERR_CUDA;          // the staging buffer may still be read by earlier work
+    for (int i = 0; i < n_chunks;) {
+        const Slice s = next_slice(descs_host, n_chunks, i, pool->n_layers, pool->n_channels, slice_bytes);
+        if (cudaMemcpyAsync(static_cast<uint8_t *>(dev_staging) + s.off,
+                            static_cast<const uint8_t *>(host_streams) + s.off, s.bytes,
+                            cudaMemcpyHostToDevice, cp) != cudaSuccess || !chain(cp, st))
+            return KVH_ERR_CUDA;
+        DecodeParams p{};
+        p.streams = static_cast<const uint8_t *>(dev_staging);
+        p.streams_bytes = staging_bytes;
+        p.descs = descs_dev + s.first;
+        p.page_table = page_table;
+        p.page_table_len = page_table_len;
+        p.status = dev_status;
+        const kvh_status ls = launch_decode(p, pool, s.count, stream);
+        if (ls != KVH_OK) return ls;
+        i += s.count;
+    }
+    if (host_status &&
+        cudaMemcpyAsync(host_status, dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KVH_ERR_CUDA;
+    return KVH_OK;
+}
+
+kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                          const kvh_chunk_desc *descs_host, const kvh_chunk_desc *descs_dev, int n_chunks,
+                          void *dev_staging, uint64_t staging_bytes, void *host_out, int32_t *dev_status,
+                          int32_t *host_status, uint64_t slice_bytes, void *copy_stream, void *stream)
+{
+    if (!kv || !dev_staging || !host_out || !descs_host || !descs_dev || n_tokens <= 0 || !copy_stream ||
+        copy_stream == stream || (host_status && !dev_status))
+        return KVH_ERR_INVALID_ARG;
+    const kvh_status s0 = check_shape(0, n_layers, n_channels);
+    if (s0 != KVH_OK) return s0;
+    if ((int64_t)n_chunks != (n_tokens + kChunkTokens - 1) / kChunkTokens) return KVH_ERR_BAD_SHAPE;
+    if (!aligned(kv, 16) || !aligned(dev_staging, KVH_SECTION_ALIGN) || !aligned(descs_dev, 8))
+        return KVH_ERR_MISALIGNED;
+    const kvh_status cs = check_contiguous(descs_host, n_chunks, n_layers, n_channels, staging_bytes);
+    if (cs != KVH_OK) return cs;
+    if (slice_bytes == 0) slice_bytes = 64ull << 20;
+    cudaStream_t cp = static_cast<cudaStream_t>(copy_stream), st = static_cast<cudaStream_t>(stream);
+    if (!chain(cp, st)) return KVH_ERR_CUDA;          // earlier copies out of the staging buffer finish first
+    for (int i = 0; i < n_chunks;) {
+        const Slice s = next_slice(descs_host, n_chunks, i, n_layers, n_channels, slice_bytes);
+        const unsigned grid = grid_for(s.count, n_layers);
+        if (grid == 0) return KVH_ERR_BAD_SHAPE;
+        EncodeParams p{};
+        p.kv = static_cast<const uint16_t *>(kv);
+        p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+        p.descs = descs_dev;
+        p.chunk0 = s.first;
+        p.out = static_cast<uint8_t *>(dev_staging);
+        p.capacity = staging_bytes;
+        p.status = dev_status;
+        encode_kernel<<<grid, kThreads, 0, st>>>(p);
+        if (launch_status() != KVH_OK || !chain(st, cp) ||
+            cudaMemcpyAsync(static_cast<uint8_t *>(host_out) + s.off,
+                            static_cast<const uint8_t *>(dev_staging) + s.off, s.bytes,
+                            cudaMemcpyDeviceToHost, cp) != cudaSuccess)
+            return KVH_ERR_CUDA;
+        i += s.count;
+    }
+    if (host_status) {
+        if (cudaMemcpyAsync(host_status, dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return KVH_ERR_CUDA;
+    }
+    return chain(cp, st) ? KVH_OK : KVH_ERR_CUDA;     // `stream` completes after the last copy out
+}
+
 }  // extern "C"

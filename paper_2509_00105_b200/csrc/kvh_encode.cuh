@@ -20,7 +20,8 @@ struct EncodeParams {
     const uint16_t *kv;            // [l][2][N][c]
     int32_t l, c;
     int64_t N;
-    const kvh_chunk_desc *descs;   // device array, or nullptr for one level throughout
+    const kvh_chunk_desc *descs;   // device array indexed by chunk, or nullptr for one level throughout
+    int32_t chunk0;                // first chunk this launch covers
     int32_t level;                 // used when descs == nullptr
     uint64_t full_chunk_bytes;     // kvh_level_bytes(level, l, c, 256), same case
     uint8_t *out;
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams 
     const int tile = b % kTilesPerChunk;  b /= kTilesPerChunk;
     const int kv = b & 1;                 b >>= 1;
     const int layer = b % p.l;
-    const int chunk = b / p.l;
+    const int chunk = p.chunk0 + b / p.l;
 
     const int64_t tok0 = (int64_t)chunk * kChunkTokens;
     const int n_expect = (int)min((int64_t)kChunkTokens, p.N - tok0);
