@@ -81,9 +81,13 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_tma_kernel, kTmaThreads, dyn) != cudaSuccess ||
             per_sm < 1)
             return KVH_ERR_CUDA;
+        // KVH_DECODE_SCHED=static walks tiles with a fixed stride instead of pulling them through
+        // cluster launch control (a measurement aid)
+        const char *sched_env = getenv("KVH_DECODE_SCHED");
+        const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
         const int64_t resident = (int64_t)sms * per_sm;
-        const unsigned pgrid = (unsigned)(grid < resident ? grid : resident);
-        decode_tma_kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages);
+        const unsigned pgrid = sched == 1 ? grid : (unsigned)(grid < resident ? grid : resident);
+        decode_tma_kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
         return launch_status();
     }
     decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);

@@ -84,6 +84,31 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
+// Cluster launch control (sm_100): a running CTA asks the hardware for the index of a CTA of this
+// grid that has not started yet and takes over its work; the 16-byte answer arrives in shared
+// memory and completes 16 bytes of transaction on the mbarrier.  Dynamic scheduling of a persistent
+// kernel without a work counter in global memory.
+__device__ __forceinline__ void clc_try_cancel(void *response, uint64_t *bar)
+{
+    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                 ::"r"(smem_addr(response)), "r"(smem_addr(bar)) : "memory");
+}
+// Decode an answer: true and the x index of the cancelled CTA, or false if none was left.
+__device__ __forceinline__ bool clc_query(const void *response, uint32_t &ctaid_x)
+{
+    uint32_t valid, x = 0;
+    asm volatile(
+        "{\n\t.reg .pred p1;\n\t.reg .b128 resp;\n\t"
+        "ld.shared.b128 resp, [%2];\n\t"
+        "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p1, resp;\n\t"
+        "selp.u32 %1, 1, 0, p1;\n\t"
+        "@p1 clusterlaunchcontrol.query_cancel.get_first_ctaid.v4.b32.b128 {%0, _, _, _}, resp;\n\t}"
+        : "+r"(x), "=r"(valid) : "r"(smem_addr(response)) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the next answer may overwrite it
+    ctaid_x = x;
+    return valid != 0;
+}
+
 __host__ __device__ __forceinline__ uint32_t tma_stage_bytes(int c) { return (36u * (uint32_t)c + 127u) & ~127u; }
 __host__ __device__ __forceinline__ uint32_t round16(uint32_t x) { return (x + 15u) & ~15u; }
 
@@ -258,14 +283,19 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
     }
 }
 
+// sched: 0 = each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (grid = resident CTAs);
+//        1 = grid holds one CTA per tile and running CTAs pull further tiles through cluster
+//            launch control, so faster SMs take more tiles.
 __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodeParams p, const int n_chunks,
-                                                                 const int n_stages)
+                                                                 const int n_stages, const int sched)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ UnitInfo info[kMaxStages];
     __shared__ int abort_flag;
+    __shared__ __align__(16) uint4 clc_response[2];
+    __shared__ __align__(8) uint64_t clc_bar[2];
 
     const uint32_t stage_bytes = tma_stage_bytes(p.c);
     const uint32_t meta_off = 32u * p.c;
@@ -276,6 +306,8 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerThreads / 32);
         }
+        mbar_init(&clc_bar[0], 1);
+        mbar_init(&clc_bar[1], 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -320,7 +352,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             return true;
         };
 
-        for (int64_t tile_id = blockIdx.x; ok && tile_id < total_tiles; tile_id += gridDim.x) {
+        auto do_tile = [&](int64_t tile_id) {
             const int tile = (int)(tile_id % kTilesPerChunk);
             const int64_t plane_id = tile_id / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
@@ -341,10 +373,10 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                     L = layer_layout(d.level, p.c, d.n_tok);
                 }
             }
-            if (!valid) continue;
+            if (!valid) return;
             const int t0 = tile * kTileTokens;
             const int nt = min(kTileTokens, d.n_tok - t0);
-            if (nt <= 0) continue;
+            if (nt <= 0) return;
             const uint8_t *lay = p.streams + d.stream_off + (uint64_t)layer * L.layer_bytes();
             const uint8_t *meta = lay + L.meta_off(kv);
             const uint8_t *codes = lay + L.codes_off(kv);
@@ -363,6 +395,38 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                 const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * (p.c / kGroup));
                 ok = emit(b, kv, t0, nt, plane, codes + (uint64_t)t0 * p.c * b / 8, cbytes, msrc, mbytes);
             }
+        };
+
+        int64_t tile_id = blockIdx.x;
+        uint32_t query = 0;                              // answers asked for so far
+        bool asked = false;                              // one answer still outstanding
+        while (ok && tile_id < total_tiles) {
+            if (sched == 1) {                            // ask for the next tile while this one streams
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&clc_bar[query & 1], 16);
+                    clc_try_cancel(&clc_response[query & 1], &clc_bar[query & 1]);
+                }
+                asked = true;
+            }
+            do_tile(tile_id);
+            if (!ok) break;
+            if (sched == 1) {
+                uint32_t got = 0, next = 0, w = 1;
+                if (lane == 0) {
+                    w = mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &abort_flag);
+                    if (w) got = clc_query(&clc_response[query & 1], next);
+                }
+                w = __shfl_sync(0xffffffffu, w, 0);
+                got = __shfl_sync(0xffffffffu, got, 0);
+                next = __shfl_sync(0xffffffffu, next, 0);
+                if (!w) { ok = false; break; }
+                asked = false;
+                ++query;
+                if (!got) break;                         // no CTA left to take over: never ask again
+                tile_id = next;
+            } else {
+                tile_id += gridDim.x;
+            }
         }
         if (ok) ok = emit(0, 0, 0, 0, nullptr, nullptr, 0, nullptr, 0);       // end marker
         if (!ok && lane == 0) {
@@ -376,6 +440,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const uint32_t first = unit > (uint32_t)n_stages ? unit - n_stages : 0;
             for (uint32_t w = first; w < unit; ++w)
                 (void)mbar_wait(&full_bar[w % n_stages], (w / n_stages) & 1, &never);
+            if (asked) (void)mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &never);
         }
     } else {
         // ------------------------------ consumer warps ------------------------------
