@@ -2,13 +2,16 @@
 //
 // This is what the paper's executor runs when the policy decides to keep an
 // entry "in full quality" (level 0) or to compress it (levels 1..3).  One HBM
-// pass: a CTA owns one (chunk, layer, K|V, 32-token tile); every thread keeps a
-// 4-channel x 32-token column of the tile in registers, so group ranges, codes
-// and packing all come from the single read of the tile.
-//   K groups run down the column (one channel, 32 tokens): a thread reduces them
-//     alone, on order-preserving integer keys.
-//   V groups run across 8 neighbouring threads (32 channels, one token): the
-//     packed (min key, inverted max key) pair is reduced with three xor-shuffles.
+// pass: a CTA owns one (chunk, layer, K|V, 32-token tile) and the group ranges,
+// the codes and their packing all come from a single read of the tile.
+//   K groups run down a column (one channel, 32 tokens): a thread holds a
+//     4-channel x 32-token column in registers and reduces it alone.
+//   V groups run along a row (32 channels, one token): a thread holds 8
+//     channels of a row, and the 4 lanes that share a group combine their ranges
+//     with two xor-shuffles; each lane derives the reciprocal scale of every
+//     fourth row and hands it round.
+// Ranges use the packed bf16 min/max instructions, which order -0 below +0 as
+// the format's definition does.
 #pragma once
 
 #include "kvh_format.cuh"
@@ -51,87 +54,171 @@ __device__ __forceinline__ void encode_tile_raw(const uint16_t *src, uint8_t *co
     for (; v < nvec; v += kThreads) d[v] = __ldcs(s + v);
 }
 
-// Store the 4 codes of one thread for one token: 4*BITS bits at element index e (multiple of 4).
-template <int BITS>
-__device__ __forceinline__ void store_codes4(uint8_t *codes, uint64_t e, uint32_t packed)
+// ---- packed bf16 helpers -------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b)
 {
-    if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(codes + e) = packed;
-    if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(codes + (e >> 1)) = (uint16_t)packed;
-    if constexpr (BITS == 2) codes[e >> 2] = (uint8_t)packed;
+    uint32_t r;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
+{
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t swap_halves(uint32_t a) { return __byte_perm(a, 0, 0x1032); }
+
+// One element: the code of x in a group with minimum lo and reciprocal scale inv.  Adding 2^23
+// rounds (x - lo) * inv to an integer, ties to even, and leaves it in the low mantissa bits; the
+// product never reaches qmax + 1/2 (it is at most qmax * (1 + 2^-22)), so no clamp is needed.
+// keep is 0x7fffff, or 0 for a group that is stored flat (then the product may be NaN).
+__device__ __forceinline__ uint32_t code_of(float x, float lo, float inv, uint32_t keep)
+{
+    const float s = __fmul_rn(__fsub_rn(x, lo), inv);
+    return __float_as_uint(__fadd_rn(s, 8388608.0f)) & keep;
 }
 
+// lo, inv and the keep mask of a group from its metadata word
 template <int BITS>
-__device__ __forceinline__ uint32_t quantise4(uint2 x, const float (&lo)[4], const float (&inv)[4])
+__device__ __forceinline__ void group_params(uint32_t meta, float &lo, float &inv, uint32_t &keep)
 {
-    return quantise<BITS>(bf16_lo_to_f32(x.x), lo[0], inv[0]) |
-           quantise<BITS>(bf16_hi_to_f32(x.x), lo[1], inv[1]) << BITS |
-           quantise<BITS>(bf16_lo_to_f32(x.y), lo[2], inv[2]) << (2 * BITS) |
-           quantise<BITS>(bf16_hi_to_f32(x.y), lo[3], inv[3]) << (3 * BITS);
+    encode_params<BITS>(meta, lo, inv);
+    keep = inv != 0.0f ? 0x7fffffu : 0u;
 }
 
+// ---- K: one group per channel ----------------------------------------------------------------
+
 template <int BITS>
-__device__ __forceinline__ void encode_tile_quant(const uint16_t *src, uint8_t *meta, uint8_t *codes,
-                                                  int c, int kv, int tile, int nt)
+__device__ __forceinline__ void encode_tile_k(const uint16_t *src, uint8_t *meta, uint8_t *codes,
+                                              int c, int tile, int nt)
 {
-    const int C4 = c >> 2;                       // 4-channel columns per row; a multiple of 8
-    const int lane = threadIdx.x & 31;
+    const int C4 = c >> 2;                       // 4-channel columns per row
     const int t0 = tile * kTileTokens;
-    // warp-uniform trip count: the V path shuffles, so whole warps stay in the loop
-    for (int base = threadIdx.x - lane; base < C4; base += kThreads) {
-        const bool active = base + lane < C4;
-        const int cq = active ? base + lane : C4 - 1;
+    for (int cq = threadIdx.x; cq < C4; cq += kThreads) {
         uint2 x[kTileTokens];
 #pragma unroll
         for (int t = 0; t < kTileTokens; ++t) {
             const int row = t < nt ? t : nt - 1;         // short tile: repeat the last valid row
             x[t] = __ldcs(reinterpret_cast<const uint2 *>(src + (uint64_t)row * c) + cq);
         }
-        if (kv == 0) {
-            // ---- K: one group per channel, down the column ----
-            uint32_t mn01 = 0xffffffffu, mn23 = 0xffffffffu, mx01 = 0, mx23 = 0;
+        uint32_t mn01 = x[0].x, mn23 = x[0].y, mx01 = x[0].x, mx23 = x[0].y;
 #pragma unroll
-            for (int t = 0; t < kTileTokens; ++t) {
-                const uint32_t k01 = order_keys2(x[t].x), k23 = order_keys2(x[t].y);
-                mn01 = __vminu2(mn01, k01); mx01 = __vmaxu2(mx01, k01);
-                mn23 = __vminu2(mn23, k23); mx23 = __vmaxu2(mx23, k23);
+        for (int t = 1; t < kTileTokens; ++t) {
+            mn01 = bmin2(mn01, x[t].x); mx01 = bmax2(mx01, x[t].x);
+            mn23 = bmin2(mn23, x[t].y); mx23 = bmax2(mx23, x[t].y);
+        }
+        // metadata words: (min | max << 16) per channel
+        const uint32_t m[4] = {__byte_perm(mn01, mx01, 0x5410), __byte_perm(mn01, mx01, 0x7632),
+                               __byte_perm(mn23, mx23, 0x5410), __byte_perm(mn23, mx23, 0x7632)};
+        float lo[4], inv[4];
+        uint32_t keep[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) group_params<BITS>(m[i], lo[i], inv[i], keep[i]);
+        *reinterpret_cast<uint4 *>(meta + 4 * ((uint64_t)tile * c + 4 * cq)) = make_uint4(m[0], m[1], m[2], m[3]);
+        uint8_t *out = codes + ((uint64_t)t0 * c + 4 * cq) * BITS / 8;
+        const uint32_t row_bytes = (uint32_t)c * BITS / 8;
+#pragma unroll
+        for (int t = 0; t < kTileTokens; ++t) {
+            if (t < nt) {
+                const uint32_t q0 = code_of(bf16_lo_to_f32(x[t].x), lo[0], inv[0], keep[0]);
+                const uint32_t q1 = code_of(bf16_hi_to_f32(x[t].x), lo[1], inv[1], keep[1]);
+                const uint32_t q2 = code_of(bf16_lo_to_f32(x[t].y), lo[2], inv[2], keep[2]);
+                const uint32_t q3 = code_of(bf16_hi_to_f32(x[t].y), lo[3], inv[3], keep[3]);
+                const uint32_t packed = (q0 + (q1 << BITS)) + ((q2 + (q3 << BITS)) << (2 * BITS));
+                if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(out) = packed;
+                if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(out) = (uint16_t)packed;
+                if constexpr (BITS == 2) *out = (uint8_t)packed;
+                out += row_bytes;
             }
-            uint32_t m[4];
-            m[0] = key_to_bf16(mn01 & 0xffffu) | key_to_bf16(mx01 & 0xffffu) << 16;
-            m[1] = key_to_bf16(mn01 >> 16) | key_to_bf16(mx01 >> 16) << 16;
-            m[2] = key_to_bf16(mn23 & 0xffffu) | key_to_bf16(mx23 & 0xffffu) << 16;
-            m[3] = key_to_bf16(mn23 >> 16) | key_to_bf16(mx23 >> 16) << 16;
-            float lo[4], inv[4];
+        }
+    }
+}
+
+// ---- V: one group per token and 32 channels --------------------------------------------------
+
+template <int BITS>
+__device__ __forceinline__ void encode_tile_v(const uint16_t *src, uint8_t *meta, uint8_t *codes,
+                                              int c, int tile, int nt)
+{
+    const int V8 = c >> 3;                               // 8-channel vectors per row, a multiple of 4
+    const int cstep = V8 <= kThreads ? V8 : kThreads;
+    const int rpp = V8 <= kThreads ? kThreads / V8 : 1;   // rows the CTA covers per pass
+    const int my_row = threadIdx.x / cstep;
+    const int my_cv = threadIdx.x - my_row * cstep;
+    if (my_row >= rpp) return;                           // whole quads of lanes leave together
+    const int lane = threadIdx.x & 31;
+    const uint32_t quad = 0xfu << (lane & ~3);           // the 4 lanes that share each group
+    const int t0 = tile * kTileTokens;
+    const int groups = c / kGroup;
+    constexpr int U = 8;                                 // rows in flight per thread
+
+    for (int cv = my_cv; cv < V8; cv += cstep) {
+        for (int tb = my_row; tb < nt; tb += U * rpp) {
+            uint4 x[U];
+            uint32_t m[U];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) encode_params<BITS>(m[i], lo[i], inv[i]);
-            if (active) {
-                *reinterpret_cast<uint4 *>(meta + 4 * ((uint64_t)tile * c + 4 * cq)) =
-                    make_uint4(m[0], m[1], m[2], m[3]);
-#pragma unroll
-                for (int t = 0; t < kTileTokens; ++t)
-                    if (t < nt)
-                        store_codes4<BITS>(codes, (uint64_t)(t0 + t) * c + 4 * cq,
-                                           quantise4<BITS>(x[t], lo, inv));
+            for (int u = 0; u < U; ++u) {
+                const int t = tb + u * rpp;
+                if (t < nt) x[u] = __ldcs(reinterpret_cast<const uint4 *>(src + (uint64_t)t * c) + cv);
             }
-        } else {
-            // ---- V: one group per token and 32 channels = 8 neighbouring lanes ----
 #pragma unroll
-            for (int t = 0; t < kTileTokens; ++t) {
-                const uint32_t k01 = order_keys2(x[t].x), k23 = order_keys2(x[t].y);
-                const uint32_t mn2 = __vminu2(k01, k23), mx2 = __vmaxu2(k01, k23);
-                // pack (min key, ~max key) so one unsigned halfword-min reduces both
-                uint32_t pk = min(mn2 & 0xffffu, mn2 >> 16) |
-                              (0xffffu - max(mx2 & 0xffffu, mx2 >> 16)) << 16;
-                pk = __vminu2(pk, __shfl_xor_sync(0xffffffffu, pk, 1));
-                pk = __vminu2(pk, __shfl_xor_sync(0xffffffffu, pk, 2));
-                pk = __vminu2(pk, __shfl_xor_sync(0xffffffffu, pk, 4));
-                const uint32_t m = key_to_bf16(pk & 0xffffu) | key_to_bf16(0xffffu - (pk >> 16)) << 16;
-                if (active && t < nt) {
-                    float l1, i1;
-                    encode_params<BITS>(m, l1, i1);
-                    const float lo[4] = {l1, l1, l1, l1}, inv[4] = {i1, i1, i1, i1};
-                    if ((cq & 7) == 0)
-                        reinterpret_cast<uint32_t *>(meta)[(uint64_t)(t0 + t) * (c / kGroup) + (cq >> 3)] = m;
-                    store_codes4<BITS>(codes, (uint64_t)(t0 + t) * c + 4 * cq, quantise4<BITS>(x[t], lo, inv));
+            for (int u = 0; u < U; ++u) {
+                if (tb + u * rpp < nt) {                 // the same for the 4 lanes of a quad
+                    uint32_t mn = bmin2(bmin2(x[u].x, x[u].y), bmin2(x[u].z, x[u].w));
+                    uint32_t mx = bmax2(bmax2(x[u].x, x[u].y), bmax2(x[u].z, x[u].w));
+                    mn = bmin2(mn, __shfl_xor_sync(quad, mn, 1));
+                    mx = bmax2(mx, __shfl_xor_sync(quad, mx, 1));
+                    mn = bmin2(mn, __shfl_xor_sync(quad, mn, 2));
+                    mx = bmax2(mx, __shfl_xor_sync(quad, mx, 2));
+                    mn = bmin2(mn, swap_halves(mn));
+                    mx = bmax2(mx, swap_halves(mx));
+                    m[u] = __byte_perm(mn, mx, 0x5410);
+                }
+            }
+            // each lane of a quad divides for every fourth row: a quarter of a division per row
+            float mine[U / 4];
+#pragma unroll
+            for (int j = 0; j < U / 4; ++j) {
+                mine[j] = 0.0f;
+                if (tb + (4 * j + (lane & 3)) * rpp < nt) {
+                    uint32_t w = m[4 * j];
+                    if ((lane & 3) == 1) w = m[4 * j + 1];
+                    if ((lane & 3) == 2) w = m[4 * j + 2];
+                    if ((lane & 3) == 3) w = m[4 * j + 3];
+                    float unused;
+                    encode_params<BITS>(w, unused, mine[j]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int t = tb + u * rpp;
+                if (t < nt) {
+                    const float inv = __shfl_sync(quad, mine[u >> 2], (lane & ~3) | (u & 3));
+                    const float lo = bf16_lo_to_f32(m[u]);
+                    const uint32_t keep = inv != 0.0f ? 0x7fffffu : 0u;
+                    const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+                    uint32_t q[8];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        q[2 * i] = code_of(bf16_lo_to_f32(w[i]), lo, inv, keep);
+                        q[2 * i + 1] = code_of(bf16_hi_to_f32(w[i]), lo, inv, keep);
+                    }
+                    const uint64_t e = (uint64_t)(t0 + t) * c + 8 * cv;
+                    if constexpr (BITS == 8) {
+                        const uint32_t a = (q[0] + (q[1] << 8)) + ((q[2] + (q[3] << 8)) << 16);
+                        const uint32_t b = (q[4] + (q[5] << 8)) + ((q[6] + (q[7] << 8)) << 16);
+                        *reinterpret_cast<uint2 *>(codes + e) = make_uint2(a, b);
+                    } else {
+                        const uint32_t a = (q[0] + (q[1] << BITS)) + ((q[2] + (q[3] << BITS)) << (2 * BITS));
+                        const uint32_t b = (q[4] + (q[5] << BITS)) + ((q[6] + (q[7] << BITS)) << (2 * BITS));
+                        const uint32_t packed = a + (b << (4 * BITS));
+                        if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(codes + (e >> 1)) = packed;
+                        if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(codes + (e >> 2)) = (uint16_t)packed;
+                    }
+                    if ((cv & 3) == 0)
+                        reinterpret_cast<uint32_t *>(meta)[(uint64_t)(t0 + t) * groups + (cv >> 2)] = m[u];
                 }
             }
         }
@@ -177,11 +264,14 @@ __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams 
         if (d.level > 0)
             zero_pad(meta, kv ? L.vmeta_payload : L.kmeta_payload, kv ? L.vmeta : L.kmeta);
     }
-    switch (d.level) {                                    // uniform per CTA
-    case 0: encode_tile_raw(src, codes, p.c, tile * kTileTokens, nt); break;
-    case 1: encode_tile_quant<8>(src, meta, codes, p.c, kv, tile, nt); break;
-    case 2: encode_tile_quant<4>(src, meta, codes, p.c, kv, tile, nt); break;
-    default: encode_tile_quant<2>(src, meta, codes, p.c, kv, tile, nt); break;
+    switch (d.level * 2 + kv) {                           // uniform per CTA
+    case 0: case 1: encode_tile_raw(src, codes, p.c, tile * kTileTokens, nt); break;
+    case 2: encode_tile_k<8>(src, meta, codes, p.c, tile, nt); break;
+    case 3: encode_tile_v<8>(src, meta, codes, p.c, tile, nt); break;
+    case 4: encode_tile_k<4>(src, meta, codes, p.c, tile, nt); break;
+    case 5: encode_tile_v<4>(src, meta, codes, p.c, tile, nt); break;
+    case 6: encode_tile_k<2>(src, meta, codes, p.c, tile, nt); break;
+    default: encode_tile_v<2>(src, meta, codes, p.c, tile, nt); break;
     }
 }
 

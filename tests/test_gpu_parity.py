@@ -68,6 +68,15 @@ def special_values(kv_np: np.ndarray, seed: int) -> None:
         kv_np[0, 0, :, 3] = rng.integers(0, 0x80, size=N)            # subnormal K channel: range < 2^-100
         kv_np[0, 1, 1, :32] = rng.choice(np.array([0x7F00, 0xFF00], dtype=np.uint16), size=32)  # +-1.7e38: range overflows
         kv_np[0, 0, :, 4] = rng.choice(np.array([0x0D80, 0x0E00, 0x0E80], dtype=np.uint16), size=N)  # range near 2^-100
+        # groups made of signed zeros only: the minimum must be -0 and the maximum +0 when both occur
+        kv_np[0, 0, :, 5] = rng.choice(np.array([0x0000, 0x8000], dtype=np.uint16), size=N)
+        kv_np[0, 0, :, 6] = np.where(np.arange(N) % 2 == 0, 0x8000, 0x0000)
+        kv_np[0, 0, :, 7] = np.where(np.arange(N) % 2 == 0, 0x0000, 0x8000)
+        if N >= 6:
+            kv_np[0, 1, 5, :32] = rng.choice(np.array([0x0000, 0x8000], dtype=np.uint16), size=32)
+        if N >= 5:
+            kv_np[0, 1, 3, :32] = np.where(np.arange(32) % 2 == 0, 0x8000, 0x0000)
+            kv_np[0, 1, 4, :32] = np.where(np.arange(32) % 2 == 0, 0x0000, 0x8000)
 
 
 SHAPES = [
