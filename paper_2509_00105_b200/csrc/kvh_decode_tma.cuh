@@ -140,20 +140,22 @@ __device__ __forceinline__ void spread8(const uint8_t *src, float (&x)[8])
     constexpr uint32_t magic = 0x4b000000u;
     uint32_t m[8];
     if constexpr (BITS == 2) {
+        // (w | magic) & (field | magic) == (w & field) | magic since w has no bit in common with
+        // magic: one logic op per code with a single immediate
         const uint32_t w = *reinterpret_cast<const uint16_t *>(src);
-        const uint32_t t = w >> 8;
+        const uint32_t wm = w | magic, tm = (w >> 8) | magic;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            m[i] = (w & (3u << (2 * i))) | magic;
-            m[i + 4] = (t & (3u << (2 * i))) | magic;
+            m[i] = wm & ((3u << (2 * i)) | magic);
+            m[i + 4] = tm & ((3u << (2 * i)) | magic);
         }
     } else if constexpr (BITS == 4) {
         const uint32_t w = *reinterpret_cast<const uint32_t *>(src);
-        const uint32_t t = w >> 16;
+        const uint32_t wm = (w & 0xffffu) | magic, tm = (w >> 16) | magic;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            m[i] = (w & (15u << (4 * i))) | magic;
-            m[i + 4] = (t & (15u << (4 * i))) | magic;
+            m[i] = wm & ((15u << (4 * i)) | magic);
+            m[i + 4] = tm & ((15u << (4 * i)) | magic);
         }
     } else {
         const uint2 w = *reinterpret_cast<const uint2 *>(src);
@@ -231,7 +233,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     const uint32_t row_bytes = (uint32_t)p.c * BITS / 8;
     const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
     uint16_t *dst = r.dst;
-#pragma unroll 2
+#pragma unroll 4
     for (int k = 0; k < r.count; ++k) {
         float x[8], f[8];
         spread8<BITS>(src, x);

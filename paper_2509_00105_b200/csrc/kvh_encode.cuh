@@ -4,8 +4,9 @@
 // entry "in full quality" (level 0) or to compress it (levels 1..3).  One HBM
 // pass: a CTA owns one (chunk, layer, K|V, 32-token tile) and the group ranges,
 // the codes and their packing all come from a single read of the tile.
-//   K groups run down a column (one channel, 32 tokens): a thread holds a
-//     4-channel x 32-token column in registers and reduces it alone.
+//   K groups run down a column (one channel, 32 tokens): two threads hold the
+//     upper and lower 16 tokens of a 4-channel column in registers and swap their
+//     partial ranges through shared memory.
 //   V groups run along a row (32 channels, one token): a thread holds 8
 //     channels of a row, and the 4 lanes that share a group combine their ranges
 //     with two xor-shuffles; each lane derives the reciprocal scale of every
@@ -70,68 +71,115 @@ __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
 }
 __device__ __forceinline__ uint32_t swap_halves(uint32_t a) { return __byte_perm(a, 0, 0x1032); }
 
-// One element: the code of x in a group with minimum lo and reciprocal scale inv.  Adding 2^23
-// rounds (x - lo) * inv to an integer, ties to even, and leaves it in the low mantissa bits; the
-// product never reaches qmax + 1/2 (it is at most qmax * (1 + 2^-22)), so no clamp is needed.
-// keep is 0x7fffff, or 0 for a group that is stored flat (then the product may be NaN).
-__device__ __forceinline__ uint32_t code_of(float x, float lo, float inv, uint32_t keep)
+// One element: 2^23 + code, as raw float bits.  Adding 2^23 rounds (x - lo) * inv to an integer,
+// ties to even, and leaves it in the low mantissa bits; the product never reaches qmax + 1/2 (it
+// is at most qmax * (1 + 2^-22)), so no clamp is needed.
+__device__ __forceinline__ uint32_t biased_code(float x, float lo, float inv)
 {
-    const float s = __fmul_rn(__fsub_rn(x, lo), inv);
-    return __float_as_uint(__fadd_rn(s, 8388608.0f)) & keep;
+    return __float_as_uint(__fadd_rn(__fmul_rn(__fsub_rn(x, lo), inv), 8388608.0f));
 }
 
-// lo, inv and the keep mask of a group from its metadata word
+// Pack 4 biased codes (0x4b000000 + q) of BITS bits: the biases add up to a constant that is
+// subtracted once, so no code is masked on its own.  Arithmetic is modulo 2^32.
 template <int BITS>
-__device__ __forceinline__ void group_params(uint32_t meta, float &lo, float &inv, uint32_t &keep)
+__device__ __forceinline__ uint32_t pack4_biased(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3)
 {
-    encode_params<BITS>(meta, lo, inv);
-    keep = inv != 0.0f ? 0x7fffffu : 0u;
+    constexpr uint32_t bias = 0x4b000000u * (1u + (1u << BITS) + (1u << (2 * BITS)) + (1u << (3 * BITS)));
+    return (t0 + (t1 << BITS)) + ((t2 + (t3 << BITS)) << (2 * BITS)) - bias;
+}
+
+// bf16 halves of a packed pair as floats; with MASKED the value of a channel whose group is
+// stored flat is replaced by 0, which makes (0 - lo) * 0 a zero and the code 0 (x - lo may
+// overflow to infinity for such a group, and infinity * 0 would be NaN).
+template <bool MASKED>
+__device__ __forceinline__ float lo_half(uint32_t pair, uint32_t mask)
+{
+    const uint32_t v = pair << 16;
+    return __uint_as_float(MASKED ? (v & mask) : v);
+}
+template <bool MASKED>
+__device__ __forceinline__ float hi_half(uint32_t pair, uint32_t mask)
+{
+    return __uint_as_float(MASKED ? (pair & 0xffff0000u & mask) : (pair & 0xffff0000u));
 }
 
 // ---- K: one group per channel ----------------------------------------------------------------
 
+constexpr int kHalfRows = kTileTokens / 2;       // rows a thread keeps in registers
+constexpr int kColThreads = kThreads / 2;        // 4-channel columns a CTA covers per pass
+
+template <int BITS, bool MASKED>
+__device__ __forceinline__ void quantise_column(const uint2 (&x)[kHalfRows], const float (&lo)[4],
+                                                const float (&inv)[4], const uint32_t (&mask)[4],
+                                                uint8_t *out, uint32_t row_bytes, int rows)
+{
+#pragma unroll
+    for (int t = 0; t < kHalfRows; ++t) {
+        if (t < rows) {
+            const uint32_t packed = pack4_biased<BITS>(
+                biased_code(lo_half<MASKED>(x[t].x, mask[0]), lo[0], inv[0]),
+                biased_code(hi_half<MASKED>(x[t].x, mask[1]), lo[1], inv[1]),
+                biased_code(lo_half<MASKED>(x[t].y, mask[2]), lo[2], inv[2]),
+                biased_code(hi_half<MASKED>(x[t].y, mask[3]), lo[3], inv[3]));
+            if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(out) = packed;
+            if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(out) = (uint16_t)packed;
+            if constexpr (BITS == 2) *out = (uint8_t)packed;
+            out += row_bytes;
+        }
+    }
+}
+
+// The CTA's two halves of 128 threads take rows 0..15 and 16..31 of a 4-channel column each, so
+// a thread keeps 16 rows in registers; the halves swap their partial ranges through shared memory.
 template <int BITS>
 __device__ __forceinline__ void encode_tile_k(const uint16_t *src, uint8_t *meta, uint8_t *codes,
-                                              int c, int tile, int nt)
+                                              int c, int tile, int nt, uint4 (*xchg)[kThreads])
 {
     const int C4 = c >> 2;                       // 4-channel columns per row
-    const int t0 = tile * kTileTokens;
-    for (int cq = threadIdx.x; cq < C4; cq += kThreads) {
-        uint2 x[kTileTokens];
+    const int half = threadIdx.x / kColThreads;
+    const int col = threadIdx.x - half * kColThreads;
+    const int r0 = half * kHalfRows;
+    const int rows = max(0, min(kHalfRows, nt - r0));    // rows of mine that exist
+    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
+    int pass = 0;
+    for (int cb = 0; cb < C4; cb += kColThreads, ++pass) {       // same trip count for every thread
+        const bool active = cb + col < C4;
+        const int cq = active ? cb + col : C4 - 1;
+        uint2 x[kHalfRows];
 #pragma unroll
-        for (int t = 0; t < kTileTokens; ++t) {
-            const int row = t < nt ? t : nt - 1;         // short tile: repeat the last valid row
+        for (int t = 0; t < kHalfRows; ++t) {
+            const int row = min(r0 + t, nt - 1);         // rows past the tile repeat its last row
             x[t] = __ldcs(reinterpret_cast<const uint2 *>(src + (uint64_t)row * c) + cq);
         }
         uint32_t mn01 = x[0].x, mn23 = x[0].y, mx01 = x[0].x, mx23 = x[0].y;
 #pragma unroll
-        for (int t = 1; t < kTileTokens; ++t) {
+        for (int t = 1; t < kHalfRows; ++t) {
             mn01 = bmin2(mn01, x[t].x); mx01 = bmax2(mx01, x[t].x);
             mn23 = bmin2(mn23, x[t].y); mx23 = bmax2(mx23, x[t].y);
         }
+        xchg[pass & 1][threadIdx.x] = make_uint4(mn01, mn23, mx01, mx23);
+        __syncthreads();
+        const uint4 o = xchg[pass & 1][threadIdx.x ^ kColThreads];
+        mn01 = bmin2(mn01, o.x); mn23 = bmin2(mn23, o.y);
+        mx01 = bmax2(mx01, o.z); mx23 = bmax2(mx23, o.w);
         // metadata words: (min | max << 16) per channel
         const uint32_t m[4] = {__byte_perm(mn01, mx01, 0x5410), __byte_perm(mn01, mx01, 0x7632),
                                __byte_perm(mn23, mx23, 0x5410), __byte_perm(mn23, mx23, 0x7632)};
         float lo[4], inv[4];
-        uint32_t keep[4];
+        uint32_t mask[4];
+        bool all_quantised = true;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) group_params<BITS>(m[i], lo[i], inv[i], keep[i]);
-        *reinterpret_cast<uint4 *>(meta + 4 * ((uint64_t)tile * c + 4 * cq)) = make_uint4(m[0], m[1], m[2], m[3]);
-        uint8_t *out = codes + ((uint64_t)t0 * c + 4 * cq) * BITS / 8;
-        const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-#pragma unroll
-        for (int t = 0; t < kTileTokens; ++t) {
-            if (t < nt) {
-                const uint32_t q0 = code_of(bf16_lo_to_f32(x[t].x), lo[0], inv[0], keep[0]);
-                const uint32_t q1 = code_of(bf16_hi_to_f32(x[t].x), lo[1], inv[1], keep[1]);
-                const uint32_t q2 = code_of(bf16_lo_to_f32(x[t].y), lo[2], inv[2], keep[2]);
-                const uint32_t q3 = code_of(bf16_hi_to_f32(x[t].y), lo[3], inv[3], keep[3]);
-                const uint32_t packed = (q0 + (q1 << BITS)) + ((q2 + (q3 << BITS)) << (2 * BITS));
-                if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(out) = packed;
-                if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(out) = (uint16_t)packed;
-                if constexpr (BITS == 2) *out = (uint8_t)packed;
-                out += row_bytes;
-            }
+        for (int i = 0; i < 4; ++i) {
+            encode_params<BITS>(m[i], lo[i], inv[i]);
+            mask[i] = inv[i] != 0.0f ? 0xffffffffu : 0u;
+            all_quantised = all_quantised && inv[i] != 0.0f;
+        }
+        if (active) {
+            if (half == 0)
+                *reinterpret_cast<uint4 *>(meta + 4 * ((uint64_t)tile * c + 4 * cq)) = make_uint4(m[0], m[1], m[2], m[3]);
+            uint8_t *out = codes + ((uint64_t)(tile * kTileTokens + r0) * c + 4 * cq) * BITS / 8;
+            if (all_quantised) quantise_column<BITS, false>(x, lo, inv, mask, out, row_bytes, rows);
+            else quantise_column<BITS, true>(x, lo, inv, mask, out, row_bytes, rows);
         }
     }
 }
@@ -197,26 +245,23 @@ __device__ __forceinline__ void encode_tile_v(const uint16_t *src, uint8_t *meta
                 if (t < nt) {
                     const float inv = __shfl_sync(quad, mine[u >> 2], (lane & ~3) | (u & 3));
                     const float lo = bf16_lo_to_f32(m[u]);
-                    const uint32_t keep = inv != 0.0f ? 0x7fffffu : 0u;
-                    const uint32_t w[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-                    uint32_t q[8];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        q[2 * i] = code_of(bf16_lo_to_f32(w[i]), lo, inv, keep);
-                        q[2 * i + 1] = code_of(bf16_hi_to_f32(w[i]), lo, inv, keep);
+                    uint32_t a = 0, b = 0;               // a flat group: every code is 0
+                    if (inv != 0.0f) {
+                        a = pack4_biased<BITS>(biased_code(lo_half<false>(x[u].x, 0), lo, inv),
+                                               biased_code(hi_half<false>(x[u].x, 0), lo, inv),
+                                               biased_code(lo_half<false>(x[u].y, 0), lo, inv),
+                                               biased_code(hi_half<false>(x[u].y, 0), lo, inv));
+                        b = pack4_biased<BITS>(biased_code(lo_half<false>(x[u].z, 0), lo, inv),
+                                               biased_code(hi_half<false>(x[u].z, 0), lo, inv),
+                                               biased_code(lo_half<false>(x[u].w, 0), lo, inv),
+                                               biased_code(hi_half<false>(x[u].w, 0), lo, inv));
                     }
                     const uint64_t e = (uint64_t)(t0 + t) * c + 8 * cv;
-                    if constexpr (BITS == 8) {
-                        const uint32_t a = (q[0] + (q[1] << 8)) + ((q[2] + (q[3] << 8)) << 16);
-                        const uint32_t b = (q[4] + (q[5] << 8)) + ((q[6] + (q[7] << 8)) << 16);
-                        *reinterpret_cast<uint2 *>(codes + e) = make_uint2(a, b);
-                    } else {
-                        const uint32_t a = (q[0] + (q[1] << BITS)) + ((q[2] + (q[3] << BITS)) << (2 * BITS));
-                        const uint32_t b = (q[4] + (q[5] << BITS)) + ((q[6] + (q[7] << BITS)) << (2 * BITS));
-                        const uint32_t packed = a + (b << (4 * BITS));
-                        if constexpr (BITS == 4) *reinterpret_cast<uint32_t *>(codes + (e >> 1)) = packed;
-                        if constexpr (BITS == 2) *reinterpret_cast<uint16_t *>(codes + (e >> 2)) = (uint16_t)packed;
-                    }
+                    if constexpr (BITS == 8) *reinterpret_cast<uint2 *>(codes + e) = make_uint2(a, b);
+                    if constexpr (BITS == 4)
+                        *reinterpret_cast<uint32_t *>(codes + (e >> 1)) = (a & 0xffffu) | (b << 16);
+                    if constexpr (BITS == 2)
+                        *reinterpret_cast<uint16_t *>(codes + (e >> 2)) = (uint16_t)((a & 0xffu) | (b << 8));
                     if ((cv & 3) == 0)
                         reinterpret_cast<uint32_t *>(meta)[(uint64_t)(t0 + t) * groups + (cv >> 2)] = m[u];
                 }
@@ -227,6 +272,7 @@ __device__ __forceinline__ void encode_tile_v(const uint16_t *src, uint8_t *meta
 
 __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams p)
 {
+    __shared__ uint4 xchg[2][kThreads];                   // K: partial ranges of the two row halves
     uint32_t b = blockIdx.x;
     const int tile = b % kTilesPerChunk;  b /= kTilesPerChunk;
     const int kv = b & 1;                 b >>= 1;
@@ -266,11 +312,11 @@ __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams 
     }
     switch (d.level * 2 + kv) {                           // uniform per CTA
     case 0: case 1: encode_tile_raw(src, codes, p.c, tile * kTileTokens, nt); break;
-    case 2: encode_tile_k<8>(src, meta, codes, p.c, tile, nt); break;
+    case 2: encode_tile_k<8>(src, meta, codes, p.c, tile, nt, xchg); break;
     case 3: encode_tile_v<8>(src, meta, codes, p.c, tile, nt); break;
-    case 4: encode_tile_k<4>(src, meta, codes, p.c, tile, nt); break;
+    case 4: encode_tile_k<4>(src, meta, codes, p.c, tile, nt, xchg); break;
     case 5: encode_tile_v<4>(src, meta, codes, p.c, tile, nt); break;
-    case 6: encode_tile_k<2>(src, meta, codes, p.c, tile, nt); break;
+    case 6: encode_tile_k<2>(src, meta, codes, p.c, tile, nt, xchg); break;
     default: encode_tile_v<2>(src, meta, codes, p.c, tile, nt); break;
     }
 }
