@@ -77,8 +77,10 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         int stages = (int)((112u * 1024u) / stage);           // two CTAs per SM when c = 1024
         stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
         const size_t dyn = (size_t)stages * stage;
-        if (cudaFuncSetAttribute(decode_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_tma_kernel, kTmaThreads, dyn) != cudaSuccess ||
+        // the instance with the channel count of the Llama-3 shapes compiled in, or the general one
+        auto kernel = p.c == 1024 ? decode_tma_kernel<1024> : decode_tma_kernel<0>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kTmaThreads, dyn) != cudaSuccess ||
             per_sm < 1)
             return KVH_ERR_CUDA;
         // KVH_DECODE_SCHED=static walks tiles with a fixed stride instead of pulling them through
@@ -87,7 +89,7 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
         const int64_t resident = (int64_t)sms * per_sm;
         const unsigned pgrid = sched == 1 ? grid : (unsigned)(grid < resident ? grid : resident);
-        decode_tma_kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
+        kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
         return launch_status();
     }
     decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);

@@ -71,13 +71,14 @@ __device__ __forceinline__ uint64_t load_codes8(const uint8_t *codes, uint64_t e
 }
 
 // Destination row of chunk token T for this plane, or nullptr if its page id is out of range.
+template <int C = 0>
 __device__ __forceinline__ uint16_t *page_row(const DecodeParams &p, int32_t pg, uint16_t *plane, int T)
 {
     if ((uint32_t)pg >= (uint32_t)p.num_pages) {
         report(p.status, KVH_ERR_PAGE_OOB);
         return nullptr;
     }
-    return plane + (int64_t)pg * p.page_stride + (int64_t)(T & (p.page_tokens - 1)) * p.c;
+    return plane + (int64_t)pg * p.page_stride + (int64_t)(T & (p.page_tokens - 1)) * (C ? C : p.c);
 }
 
 template <int BITS>

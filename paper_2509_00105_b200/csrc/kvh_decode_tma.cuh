@@ -182,9 +182,10 @@ struct RowRun {
     uint16_t *dst;              // first row's destination (already offset by cv), nullptr if none
 };
 
+template <int C>
 __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u)
 {
-    const int V8 = p.c >> 3;                              // <= 128
+    const int V8 = (C ? C : p.c) >> 3;                              // <= 128
     const int rpp = kConsumerThreads / V8;                // row groups the CTA holds, >= 2
     int rpt = 1;
     while (rpt * rpp < kTileTokens) rpt <<= 1;            // rows per thread: 16 when c = 1024
@@ -197,27 +198,30 @@ __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo 
     if (r.count > 0) {
         const int T = u.row0 + r.first;
         const int32_t pg = (T >> p.page_shift) == (u.row0 >> p.page_shift) ? u.pg0 : u.pg1;
-        r.dst = page_row(p, pg, u.plane, T);              // reports an out-of-range page id
+        r.dst = page_row<C>(p, pg, u.plane, T);              // reports an out-of-range page id
         if (r.dst) r.dst += 8 * r.cv; else r.count = 0;
     }
     return r;
 }
 
+template <int C>
 __device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
 {
-    const RowRun r = row_run(p, u);
-    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * p.c + 8 * r.cv));
+    const int c = C ? C : p.c;
+    const RowRun r = row_run<C>(p, u);
+    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * c + 8 * r.cv));
     uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
-    const int stride = p.c >> 3;                          // uint4 per row
+    const int stride = c >> 3;                            // uint4 per row
 #pragma unroll 4
     for (int k = 0; k < r.count; ++k) dst[(size_t)k * stride] = src[(size_t)k * stride];
 }
 
-template <int BITS>
+template <int BITS, int C>
 __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
-    const RowRun r = row_run(p, u);
+    const int c = C ? C : p.c;
+    const RowRun r = row_run<C>(p, u);
     if (r.count == 0) return;
     float lo[8], sc[8];
     {
@@ -230,7 +234,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
             sc[i] = __fmul_rn(sc[i], Pos<BITS>::prescale(i));
         }
     }
-    const uint32_t row_bytes = (uint32_t)p.c * BITS / 8;
+    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
     const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
     uint16_t *dst = r.dst;
 #pragma unroll 4
@@ -241,20 +245,21 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
         for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], sc[i], lo[i]);
         *reinterpret_cast<uint4 *>(dst) = pack8(f);
         src += row_bytes;
-        dst += p.c;
+        dst += c;
     }
 }
 
-template <int BITS>
+template <int BITS, int C>
 __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
-    const RowRun r = row_run(p, u);
+    const int c = C ? C : p.c;
+    const RowRun r = row_run<C>(p, u);
     const int lane = threadIdx.x & 31;
     const uint32_t quad = 0xfu << (lane & ~3);            // the 4 lanes that share every V group
-    const int groups = p.c / kGroup;
+    const int groups = c / kGroup;
     const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)r.first * groups + (r.cv >> 2);
-    const uint32_t row_bytes = (uint32_t)p.c * BITS / 8;
+    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
     const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
     uint16_t *dst = r.dst;
     // r.count is the same for the 4 lanes of a quad (they share the row group), so the shuffles
@@ -279,7 +284,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
                 for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], s[i & 3], l1);
                 *reinterpret_cast<uint4 *>(dst) = pack8(f);
                 src += row_bytes;
-                dst += p.c;
+                dst += c;
             }
         }
     }
@@ -288,6 +293,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
 // sched: 0 = each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (grid = resident CTAs);
 //        1 = grid holds one CTA per tile and running CTAs pull further tiles through cluster
 //            launch control, so faster SMs take more tiles.
+template <int C>
 __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodeParams p, const int n_chunks,
                                                                  const int n_stages, const int sched)
 {
@@ -458,13 +464,13 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const uint8_t *mt = st + meta_off;
             switch (u.bits * 2 + u.kv) {                      // uniform per CTA
-            case 32: case 33: consume_raw(p, u, st); break;
-            case 16: consume_k<8>(p, u, st, mt); break;
-            case 17: consume_v<8>(p, u, st, mt); break;
-            case 8: consume_k<4>(p, u, st, mt); break;
-            case 9: consume_v<4>(p, u, st, mt); break;
-            case 4: consume_k<2>(p, u, st, mt); break;
-            default: consume_v<2>(p, u, st, mt); break;
+            case 32: case 33: consume_raw<C>(p, u, st); break;
+            case 16: consume_k<8, C>(p, u, st, mt); break;
+            case 17: consume_v<8, C>(p, u, st, mt); break;
+            case 8: consume_k<4, C>(p, u, st, mt); break;
+            case 9: consume_v<4, C>(p, u, st, mt); break;
+            case 4: consume_k<2, C>(p, u, st, mt); break;
+            default: consume_v<2, C>(p, u, st, mt); break;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[s]);
