@@ -182,6 +182,37 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
                           int32_t *dev_status, int32_t *host_status, uint64_t slice_bytes,
                           void *copy_stream, void *stream);
 
+/* ---- a load entry point that allocates nothing -------------------------------------------------
+ *
+ * The paper has no counterpart to this call; it exists for how the library gets deployed.  Some
+ * callers of kvh_load_host have no device allocator at hand when a cache hit arrives: a plug-in
+ * running inside a serving engine that has already handed all free HBM to its paged KV pool, a
+ * thread that must not take the allocator's lock, or code running while a stream capture is open
+ * elsewhere in the process, where cudaMalloc is not permitted.  For them the staging area that
+ * kvh_load_host takes as an argument is a fixed array inside the library's device image,
+ * KVH_STATIC_STAGING_BYTES long.  Every GPU on which the library is loaded gives up that much
+ * memory until the process exits, whether or not this call is ever made.
+ *
+ * Arguments and behaviour are those of kvh_load_host without dev_staging / staging_bytes.  The
+ * descriptors' stream offsets index the host buffer and the fixed array alike, so the end of the
+ * last chunk (its stream_off plus its size) must not exceed KVH_STATIC_STAGING_BYTES; a larger
+ * request returns KVH_ERR_BUFFER_TOO_SMALL with nothing enqueued (split it into several calls
+ * whose descriptors start again at offset 0).  The call itself creates no device or host memory.
+ *
+ * The first call on each device looks up the array's device address (with that device current)
+ * and remembers it; make that first call outside any stream capture.  All calls on a device
+ * share the one array and it keeps whatever the last call left there: nothing in it needs to
+ * start at zero, because every byte a decode reads is copied in by the same call first.  Two
+ * calls whose GPU work can overlap (different `stream`s, or several host threads) overwrite each
+ * other's staged chunks; order them on one stream or with events. */
+#define KVH_STATIC_STAGING_BYTES (64u << 20)
+
+kvh_status kvh_load_host_static(const void *host_streams,
+                                const kvh_chunk_desc *descs_host, const kvh_chunk_desc *descs_dev,
+                                int n_chunks, const int32_t *page_table, int64_t page_table_len,
+                                const kvh_pool *pool, int32_t *dev_status, int32_t *host_status,
+                                uint64_t slice_bytes, void *copy_stream, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

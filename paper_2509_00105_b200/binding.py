@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
                                     u64, vp, vp]
         L.kvh_store_host.restype = i32
         L.kvh_store_host.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, u64, vp, vp, vp, u64, vp, vp]
+        L.kvh_load_host_static.restype = i32
+        L.kvh_load_host_static.argtypes = [vp, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp, u64, vp, vp]
         _lib = L
     return _lib
 
@@ -245,3 +247,25 @@ def store_host(kv: torch.Tensor, descs: np.ndarray, descs_dev: torch.Tensor, sta
                                 staging.data_ptr(), staging.numel(), host_out.data_ptr(), _ptr(dev_status),
                                 _ptr(host_status), slice_bytes, copy_stream.cuda_stream, _stream()),
            "kvh_store_host")
+
+
+STATIC_STAGING_BYTES = 64 << 20
+
+
+def load_host_static(host_streams: torch.Tensor, descs: np.ndarray, descs_dev: torch.Tensor,
+                     page_table: torch.Tensor, pool: Pool, dev_status: torch.Tensor | None,
+                     host_status: torch.Tensor | None, copy_stream: torch.cuda.Stream, slice_bytes: int = 0) -> None:
+    """load_host() for callers that cannot allocate device memory: the chunks are staged in a fixed
+    array of STATIC_STAGING_BYTES inside the library instead of a tensor of the caller's.  The
+    stream offsets in `descs` must end within that size.  Calls on one device share the array, so
+    keep them on one stream (or order them with events)."""
+    assert host_streams.is_pinned() and host_streams.dtype == torch.uint8 and descs.dtype == DESC_DTYPE
+    assert host_status is None or (host_status.is_pinned() and host_status.dtype == torch.int32)
+    need = int(descs["stream_off"][-1]) + level_bytes(int(descs["level"][-1]), pool.struct.n_layers,
+                                                       pool.struct.n_channels, int(descs["n_tok"][-1]))
+    if host_streams.numel() < need:
+        raise KvhError(5, "load_host_static")
+    _check(lib().kvh_load_host_static(host_streams.data_ptr(), descs.ctypes.data, descs_dev.data_ptr(), len(descs),
+                                      page_table.data_ptr(), page_table.numel(), ctypes.byref(pool.struct),
+                                      _ptr(dev_status), _ptr(host_status), slice_bytes, copy_stream.cuda_stream,
+                                      _stream()), "kvh_load_host_static")

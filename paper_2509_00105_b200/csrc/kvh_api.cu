@@ -393,3 +393,52 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
 }
 
 }  // extern "C"
+
+// ---- host-tier load for callers that cannot allocate device memory --------------------------
+
+namespace {
+
+// Staging area of kvh_load_host_static.  It lives in the library's device image, so every GPU
+// that loads the library sets this much memory aside until the process exits.
+static __device__ __align__(256) uint8_t g_static_staging[KVH_STATIC_STAGING_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_static_staging_ptr[kMaxDevices];      // device address of the array, per device; nullptr = not set up
+
+// g_static_staging names a host-side handle here, not device memory: the address a kernel or a
+// copy may use comes from cudaGetSymbolAddress, asked once per device with that device current.
+kvh_status static_staging_address(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return KVH_ERR_CUDA;
+    void *p = __atomic_load_n(&g_static_staging_ptr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_static_staging) != cudaSuccess || !p) return KVH_ERR_CUDA;
+        __atomic_store_n(&g_static_staging_ptr[dev], p, __ATOMIC_RELEASE);    // every thread gets the same answer
+    }
+    *out = p;
+    return KVH_OK;
+}
+
+}  // namespace
+
+extern "C" kvh_status kvh_load_host_static(const void *host_streams, const kvh_chunk_desc *descs_host,
+                                           const kvh_chunk_desc *descs_dev, int n_chunks,
+                                           const int32_t *page_table, int64_t page_table_len,
+                                           const kvh_pool *pool, int32_t *dev_status, int32_t *host_status,
+                                           uint64_t slice_bytes, void *copy_stream, void *stream)
+{
+    if (!descs_host || n_chunks <= 0) return KVH_ERR_INVALID_ARG;
+    const kvh_status ps = check_pool(pool);
+    if (ps != KVH_OK) return ps;
+    // the stored form must fit the fixed staging area: say so before anything is enqueued
+    const kvh_status cs = check_contiguous(descs_host, n_chunks, pool->n_layers, pool->n_channels,
+                                           KVH_STATIC_STAGING_BYTES);
+    if (cs != KVH_OK) return cs;                // KVH_ERR_BUFFER_TOO_SMALL: beyond KVH_STATIC_STAGING_BYTES
+    void *staging = nullptr;
+    const kvh_status as = static_staging_address(&staging);
+    if (as != KVH_OK) return as;
+    return kvh_load_host(host_streams, staging, KVH_STATIC_STAGING_BYTES, descs_host, descs_dev, n_chunks,
+                         page_table, page_table_len, pool, dev_status, host_status, slice_bytes, copy_stream,
+                         stream);
+}
