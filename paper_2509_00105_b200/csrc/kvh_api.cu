@@ -11,7 +11,12 @@
 #include "kvh_decode.cuh"
 #include "kvh_decode_tma.cuh"
 #include "kvh_encode.cuh"
+#include "kvh_encode_tma.cuh"
 #include "kvh_format.cuh"
+
+#ifndef KVH_ENCODE_GROUPS
+#define KVH_ENCODE_GROUPS 1     // consumer groups of 256 threads in the TMA-fed encode kernel
+#endif
 
 using namespace kvh;
 
@@ -93,6 +98,46 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         return launch_status();
     }
     decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return launch_status();
+}
+
+// Encode launch: the persistent TMA-fed kernel when a 32-token tile fits a shared-memory stage,
+// otherwise one CTA per tile reading global memory directly.  KVH_ENCODE_PATH=direct forces the
+// latter and KVH_ENCODE_SCHED=static a fixed tile stride (measurement aids).
+kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream)
+{
+    const unsigned grid = grid_for(n_chunks, p.l);
+    if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const char *force = getenv("KVH_ENCODE_PATH");
+    if (p.c <= kEncMaxChannels && !(force && strcmp(force, "direct") == 0)) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return KVH_ERR_CUDA;
+        constexpr int G = KVH_ENCODE_GROUPS;
+        const size_t dyn = (size_t)kEncStages * kEncStageBytes;
+        // one level for the whole launch (kvh_encode): an instance that holds only that level's code
+        const int level = p.descs ? -1 : p.level;
+        void (*kernel)(const EncodeParams, const int, const int);
+        if (p.c == 1024) {
+            kernel = level == 0 ? encode_tma_kernel<1024, G, 0> : level == 1 ? encode_tma_kernel<1024, G, 1>
+                   : level == 2 ? encode_tma_kernel<1024, G, 2> : level == 3 ? encode_tma_kernel<1024, G, 3>
+                   : encode_tma_kernel<1024, G, -1>;
+        } else {
+            kernel = level == 0 ? encode_tma_kernel<0, G, 0> : level == 1 ? encode_tma_kernel<0, G, 1>
+                   : level == 2 ? encode_tma_kernel<0, G, 2> : level == 3 ? encode_tma_kernel<0, G, 3>
+                   : encode_tma_kernel<0, G, -1>;
+        }
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+            return KVH_ERR_CUDA;
+        const char *sched_env = getenv("KVH_ENCODE_SCHED");
+        const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
+        const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
+        kernel<<<pgrid, 32 + G * kEncGroupThreads, dyn, st>>>(p, (int)n_chunks, sched);
+        return launch_status();
+    }
+    encode_kernel<<<grid, kThreads, 0, st>>>(p);
     return launch_status();
 }
 
@@ -180,8 +225,6 @@ kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_chan
     if (ps != KVH_OK) return ps;
     if (need > out_capacity) return KVH_ERR_BUFFER_TOO_SMALL;
     const int64_t n_chunks = (n_tokens + kChunkTokens - 1) / kChunkTokens;
-    const unsigned grid = grid_for(n_chunks, n_layers);
-    if (grid == 0) return KVH_ERR_BAD_SHAPE;
     EncodeParams p{};
     p.kv = static_cast<const uint16_t *>(kv);
     p.l = n_layers; p.c = n_channels; p.N = n_tokens;
@@ -191,8 +234,7 @@ kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_chan
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
     p.status = dev_status;
-    encode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
-    return launch_status();
+    return launch_encode(p, n_chunks, stream);
 }
 
 kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
@@ -204,8 +246,6 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
     if (s != KVH_OK) return s;
     if ((int64_t)n_chunks != (n_tokens + kChunkTokens - 1) / kChunkTokens) return KVH_ERR_BAD_SHAPE;
     if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
-    const unsigned grid = grid_for(n_chunks, n_layers);
-    if (grid == 0) return KVH_ERR_BAD_SHAPE;
     EncodeParams p{};
     p.kv = static_cast<const uint16_t *>(kv);
     p.l = n_layers; p.c = n_channels; p.N = n_tokens;
@@ -213,8 +253,7 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
     p.status = dev_status;
-    encode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
-    return launch_status();
+    return launch_encode(p, n_chunks, stream);
 }
 
 kvh_status kvh_decode_to_pages(const void *chunk, int level, int n_tok, const int32_t *page_ids,
@@ -367,8 +406,6 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
     if (!chain(cp, st)) return KVH_ERR_CUDA;          // earlier copies out of the staging buffer finish first
     for (int i = 0; i < n_chunks;) {
         const Slice s = next_slice(descs_host, n_chunks, i, n_layers, n_channels, slice_bytes);
-        const unsigned grid = grid_for(s.count, n_layers);
-        if (grid == 0) return KVH_ERR_BAD_SHAPE;
         EncodeParams p{};
         p.kv = static_cast<const uint16_t *>(kv);
         p.l = n_layers; p.c = n_channels; p.N = n_tokens;
@@ -377,8 +414,9 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
         p.out = static_cast<uint8_t *>(dev_staging);
         p.capacity = staging_bytes;
         p.status = dev_status;
-        encode_kernel<<<grid, kThreads, 0, st>>>(p);
-        if (launch_status() != KVH_OK || !chain(st, cp) ||
+        const kvh_status ls = launch_encode(p, s.count, st);
+        if (ls != KVH_OK) return ls;
+        if (!chain(st, cp) ||
             cudaMemcpyAsync(static_cast<uint8_t *>(host_out) + s.off,
                             static_cast<const uint8_t *>(dev_staging) + s.off, s.bytes,
                             cudaMemcpyDeviceToHost, cp) != cudaSuccess)

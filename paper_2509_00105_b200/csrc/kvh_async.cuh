@@ -1,0 +1,87 @@
+// Asynchronous-copy and scheduling primitives of sm_100 used by the persistent kernels of this
+// library: mbarriers with bounded waits, 1-D bulk copies between global and shared memory, and
+// cluster launch control (a running CTA takes over the work of CTAs that have not started yet).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kvh {
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: no wait in a kernel lasts longer
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a phase of an mbarrier; false if the time limit ran out or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long start = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag || global_ns() - start > kWaitLimitNs) return false;
+    }
+}
+// 1-D bulk copy global -> this CTA's shared memory; bytes is a multiple of 16, both ends 16-byte aligned.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// Cluster launch control (sm_100): a running CTA asks the hardware for the index of a CTA of this
+// grid that has not started yet and takes over its work; the 16-byte answer arrives in shared
+// memory and completes 16 bytes of transaction on the mbarrier.  Dynamic scheduling of a persistent
+// kernel without a work counter in global memory.
+__device__ __forceinline__ void clc_try_cancel(void *response, uint64_t *bar)
+{
+    asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                 ::"r"(smem_addr(response)), "r"(smem_addr(bar)) : "memory");
+}
+// Decode an answer: true and the x index of the cancelled CTA, or false if none was left.
+__device__ __forceinline__ bool clc_query(const void *response, uint32_t &ctaid_x)
+{
+    uint32_t valid, x = 0;
+    asm volatile(
+        "{\n\t.reg .pred p1;\n\t.reg .b128 resp;\n\t"
+        "ld.shared.b128 resp, [%2];\n\t"
+        "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p1, resp;\n\t"
+        "selp.u32 %1, 1, 0, p1;\n\t"
+        "@p1 clusterlaunchcontrol.query_cancel.get_first_ctaid.v4.b32.b128 {%0, _, _, _}, resp;\n\t}"
+        : "+r"(x), "=r"(valid) : "r"(smem_addr(response)) : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the next answer may overwrite it
+    ctaid_x = x;
+    return valid != 0;
+}
+
+}  // namespace kvh

@@ -1,0 +1,571 @@
+// Persistent, TMA-fed encode kernel (the fast path for c <= 1024).
+//
+// Storing a context is the executor's other direction: the policy has decided to keep an entry
+// "in full quality" (level 0) or to compress it (levels 1..3), and the KV tensor has to be turned
+// into chunk streams at the speed HBM delivers it (2 bytes read and (b+1)/8 bytes written per
+// element).  A 32-token tile of one (layer, K|V) plane is contiguous in the source, so a producer
+// warp brings it into a ring of 64 KiB shared-memory stages with one 1-D bulk async copy per tile
+// while 8 consumer warps turn the previous tiles into metadata and codes:
+//   K (a group = one channel over the tile's 32 tokens): a thread owns 4 channels and keeps all
+//     32 rows of them in registers, so ranges, scales and codes need one pass over shared memory
+//     and no exchange between threads.
+//   V (a group = 32 channels of one token): a thread owns whole groups (64 bytes), again with no
+//     exchange.  Neighbouring lanes are 64 bytes apart, so each lane reads its four 16-byte pieces
+//     in an order rotated by its lane number (bank conflicts vanish) and rotates the packed codes
+//     back in registers before one wide store.
+// The three roundings of a code, (x - min) * inv + 2^23, are done two elements at a time with the
+// packed binary32 instructions of sm_100 (sub/mul/fma .rn.f32x2: IEEE round-to-nearest on each
+// half, no flush to zero), which halves the issue slots the arithmetic takes.  A stage is handed
+// back to the producer as soon as its data sits in registers.
+//
+// Tiles are handed out dynamically through cluster launch control, as in the decode kernel.  Every
+// wait is bounded: when one runs out the CTA reports KVH_ERR_TIMEOUT, raises its abort flag,
+// waits for its copies in flight and leaves.
+#pragma once
+
+#include "kvh_async.cuh"
+#include "kvh_encode.cuh"
+#include "kvh_format.cuh"
+
+namespace kvh {
+
+constexpr int kEncGroupThreads = 256;                    // consumer threads that share a tile
+constexpr int kEncStages = 3;
+constexpr uint32_t kEncStageBytes = 2u * kTileTokens * 1024u;   // a 32-token tile at c = 1024
+constexpr int kEncMaxChannels = 1024;
+
+struct EncUnit {
+    int32_t bits;          // 16, 8, 4, 2; 0 marks the end of the CTA's work
+    int32_t kv;            // 0 K, 1 V
+    int32_t nt;            // tokens in the tile (1..32)
+    int32_t tile;          // tile index within the chunk
+    int32_t last;          // the plane's last tile clears the sections' padding
+    uint32_t meta_payload, meta_padded, codes_payload, codes_padded;
+    uint8_t *meta;         // the plane's metadata section in the stream
+    uint8_t *codes;        // the plane's code section
+};
+
+// ---- two binary32 values in one 64-bit register -----------------------------------------------
+
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 f2_from_bits(uint32_t a, uint32_t b)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_make(float a, float b) { return f2_from_bits(__float_as_uint(a), __float_as_uint(b)); }
+__device__ __forceinline__ void f2_bits(f32x2 v, uint32_t &a, uint32_t &b)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 f2_sub(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_mul(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_fma(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+// Both elements of a packed bf16 pair: 2^23 + code as raw float bits (see biased_code()).  With
+// MASKED the value of a channel whose group is stored flat is replaced by 0 first, so that its
+// code is 0 even when x - min overflows.
+template <bool MASKED>
+__device__ __forceinline__ void biased_pair(uint32_t w, f32x2 lo2, f32x2 inv2, uint32_t mask_a, uint32_t mask_b,
+                                            uint32_t &ta, uint32_t &tb)
+{
+    uint32_t a = w << 16, b = w & 0xffff0000u;
+    if (MASKED) { a &= mask_a; b &= mask_b; }
+    const f32x2 magic = f2_from_bits(0x4b000000u, 0x4b000000u);
+    // The product must be rounded before 2^23 is added.  A packed mul followed by a packed add gets
+    // contracted into one fused multiply-add by the assembler (even with .rn on both), which skips
+    // that rounding and moves about one code in a thousand; written as fma(s, 1, 2^23) the addition
+    // cannot absorb the multiply and rounds s + 2^23 once, exactly like an add.
+    const f32x2 s = f2_mul(f2_sub(f2_from_bits(a, b), lo2), inv2);
+    f2_bits(f2_fma(s, f2_from_bits(0x3f800000u, 0x3f800000u), magic), ta, tb);
+}
+
+// Four biased codes (0x4b000000 + q) into the low 4 * BITS bits.  For 2 and 4 bits the biases end
+// up above the field and the caller's narrow store (or a byte permute) drops them.
+template <int BITS>
+__device__ __forceinline__ uint32_t pack4_low(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3)
+{
+    if constexpr (BITS == 8) {
+        return __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+    } else {
+        return (t0 + (t1 << BITS)) + ((t2 + (t3 << BITS)) << (2 * BITS));
+    }
+}
+
+// Hand a stage back to the producer: every lane's reads of it are done.
+__device__ __forceinline__ void enc_release(uint64_t *empty_bar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(empty_bar);
+}
+
+// ---- level 0: the tile's rows as they are ------------------------------------------------------
+
+template <int C>
+__device__ __forceinline__ void enc_consume_raw(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                             int nt, int tile, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int nvec = nt * (c >> 3);
+    const uint4 *src = reinterpret_cast<const uint4 *>(st);
+    uint4 *dst = reinterpret_cast<uint4 *>(codes_sec + 2 * (size_t)tile * kTileTokens * c);
+    constexpr int U = 8;
+    const int iters = (nvec + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);     // the same for every thread
+    for (int it = 0; it < iters; ++it) {
+        const int v0 = it * kEncGroupThreads * U + tid;
+        uint4 x[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+            if (v0 + k * kEncGroupThreads < nvec) x[k] = src[v0 + k * kEncGroupThreads];
+        if (it == iters - 1) enc_release(empty_bar);
+#pragma unroll
+        for (int k = 0; k < U; ++k)
+            if (v0 + k * kEncGroupThreads < nvec) __stcs(dst + v0 + k * kEncGroupThreads, x[k]);
+    }
+}
+
+// ---- K: one group per channel -------------------------------------------------------------------
+
+// Codes of one row of a 4-channel column, stored with the width the level needs.
+template <int BITS, bool MASKED>
+__device__ __forceinline__ void enc_store_row_k(uint2 x, f32x2 lo_a, f32x2 lo_b, f32x2 inv_a, f32x2 inv_b,
+                                                const uint32_t (&mask)[4], uint8_t *o)
+{
+    uint32_t t0, t1, t2, t3;
+    biased_pair<MASKED>(x.x, lo_a, inv_a, mask[0], mask[1], t0, t1);
+    biased_pair<MASKED>(x.y, lo_b, inv_b, mask[2], mask[3], t2, t3);
+    const uint32_t packed = pack4_low<BITS>(t0, t1, t2, t3);
+    if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(o) = packed;
+    if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(o) = (uint16_t)packed;
+    if constexpr (BITS == 2) *o = (uint8_t)packed;
+}
+
+// Metadata words (min | max << 16) of 4 channels from their packed ranges, and what follows
+// from them; returns whether every one of the 4 groups is quantised (none stored flat).
+template <int BITS>
+__device__ __forceinline__ bool enc_params_k(uint32_t mn01, uint32_t mn23, uint32_t mx01, uint32_t mx23,
+                                             uint4 *meta_out, float (&lo)[4], float (&inv)[4], uint32_t (&mask)[4])
+{
+    const uint32_t m[4] = {__byte_perm(mn01, mx01, 0x5410), __byte_perm(mn01, mx01, 0x7632),
+                           __byte_perm(mn23, mx23, 0x5410), __byte_perm(mn23, mx23, 0x7632)};
+    bool all_quantised = true;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        encode_params<BITS>(m[i], lo[i], inv[i]);
+        mask[i] = inv[i] != 0.0f ? 0xffffffffu : 0u;
+        all_quantised = all_quantised && inv[i] != 0.0f;
+    }
+    *meta_out = make_uint4(m[0], m[1], m[2], m[3]);
+    return all_quantised;
+}
+
+// A full tile: all 32 rows of the thread's 4 channels in registers, one pass over shared memory.
+template <int BITS, int C>
+__device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                              int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int C4 = c >> 2;                               // 4-channel columns per row, <= 256
+    const bool active = tid < C4;
+    const int cq = active ? tid : 0;
+    const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
+    uint2 x[kTileTokens];
+#pragma unroll
+    for (int t = 0; t < kTileTokens; ++t) x[t] = col[t * C4];
+    enc_release(empty_bar);
+    if (!active) return;
+
+    uint32_t mn01 = x[0].x, mn23 = x[0].y, mx01 = x[0].x, mx23 = x[0].y;
+#pragma unroll
+    for (int t = 1; t < kTileTokens; ++t) {
+        mn01 = bmin2(mn01, x[t].x); mx01 = bmax2(mx01, x[t].x);
+        mn23 = bmin2(mn23, x[t].y); mx23 = bmax2(mx23, x[t].y);
+    }
+    float lo[4], inv[4];
+    uint32_t mask[4];
+    const bool all_quantised = enc_params_k<BITS>(
+        mn01, mn23, mx01, mx23, reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
+    if (!all_quantised) {
+        // a channel stored flat: its values become 0 so that (0 - min) * 0 is a zero and the code 0
+        // (x - min may overflow for such a group, and infinity * 0 would be NaN)
+        const uint32_t k01 = (mask[0] & 0xffffu) | (mask[1] & 0xffff0000u);
+        const uint32_t k23 = (mask[2] & 0xffffu) | (mask[3] & 0xffff0000u);
+#pragma unroll
+        for (int t = 0; t < kTileTokens; ++t) { x[t].x &= k01; x[t].y &= k23; }
+    }
+    const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
+    const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
+    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
+    uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
+#pragma unroll
+    for (int t = 0; t < kTileTokens; ++t)
+        enc_store_row_k<BITS, false>(x[t], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
+}
+
+// The last, short tile of a chunk (nt < 32 rows): rare, so two plain passes over shared memory.
+template <int BITS>
+__device__ __noinline__ void enc_consume_k_short(const uint8_t *st, int c, int tid, uint64_t *empty_bar,
+                                                 int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int C4 = c >> 2;
+    if (tid < C4) {
+        const int cq = tid;
+        const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
+        uint32_t mn01 = col[0].x, mn23 = col[0].y, mx01 = mn01, mx23 = mn23;
+#pragma unroll 1
+        for (int t = 1; t < nt; ++t) {
+            const uint2 x = col[t * C4];
+            mn01 = bmin2(mn01, x.x); mx01 = bmax2(mx01, x.x);
+            mn23 = bmin2(mn23, x.y); mx23 = bmax2(mx23, x.y);
+        }
+        float lo[4], inv[4];
+        uint32_t mask[4];
+        (void)enc_params_k<BITS>(mn01, mn23, mx01, mx23,
+                                 reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
+        const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
+        const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
+        const uint32_t row_bytes = (uint32_t)c * BITS / 8;
+        uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
+#pragma unroll 1
+        for (int t = 0; t < nt; ++t)
+            enc_store_row_k<BITS, true>(col[t * C4], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
+    }
+    enc_release(empty_bar);
+}
+
+// ---- V: one group per token and 32 channels ---------------------------------------------------
+
+// p[j] holds the piece with number (j + rot) & 3; put piece k into p[k].
+template <int W>
+__device__ __forceinline__ void enc_unrotate(uint32_t (&p)[4][W], int rot)
+{
+    const bool r1 = rot & 1, r2 = rot & 2;
+    uint32_t q[4][W];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int w = 0; w < W; ++w) q[k][w] = r1 ? p[(k + 3) & 3][w] : p[k][w];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int w = 0; w < W; ++w) p[k][w] = r2 ? q[(k + 2) & 3][w] : q[k][w];
+}
+
+// One group: range, metadata word, codes.  x[j] is the 16-byte piece number (j + rot) & 3 of the
+// group's 64 bytes.
+template <int BITS>
+__device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32_t *meta_out, uint8_t *codes_out)
+{
+    uint32_t mn = bmin2(bmin2(x[0].x, x[0].y), bmin2(x[0].z, x[0].w));
+    uint32_t mx = bmax2(bmax2(x[0].x, x[0].y), bmax2(x[0].z, x[0].w));
+#pragma unroll
+    for (int j = 1; j < 4; ++j) {
+        mn = bmin2(mn, bmin2(bmin2(x[j].x, x[j].y), bmin2(x[j].z, x[j].w)));
+        mx = bmax2(mx, bmax2(bmax2(x[j].x, x[j].y), bmax2(x[j].z, x[j].w)));
+    }
+    mn = bmin2(mn, swap_halves(mn));
+    mx = bmax2(mx, swap_halves(mx));
+    const uint32_t m = __byte_perm(mn, mx, 0x5410);
+    *meta_out = m;
+    float lo, inv;
+    encode_params<BITS>(m, lo, inv);
+    constexpr int W = BITS == 8 ? 2 : 1;                 // words a piece's 8 codes take (16 bits used at 2 bits)
+    uint32_t p[4][W];
+    if (inv != 0.0f) {
+        const f32x2 lo2 = f2_make(lo, lo), inv2 = f2_make(inv, inv);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t t[8];
+            biased_pair<false>(x[j].x, lo2, inv2, 0, 0, t[0], t[1]);
+            biased_pair<false>(x[j].y, lo2, inv2, 0, 0, t[2], t[3]);
+            biased_pair<false>(x[j].z, lo2, inv2, 0, 0, t[4], t[5]);
+            biased_pair<false>(x[j].w, lo2, inv2, 0, 0, t[6], t[7]);
+            const uint32_t a = pack4_low<BITS>(t[0], t[1], t[2], t[3]);
+            const uint32_t b = pack4_low<BITS>(t[4], t[5], t[6], t[7]);
+            if constexpr (BITS == 8) { p[j][0] = a; p[j][1] = b; }
+            if constexpr (BITS == 4) p[j][0] = __byte_perm(a, b, 0x5410);
+            if constexpr (BITS == 2) p[j][0] = __byte_perm(a, b, 0x0040);     // 16 bits; the upper half is dropped below
+        }
+        enc_unrotate<W>(p, rot);
+    } else {                                             // a flat group: every code is 0
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int w = 0; w < W; ++w) p[j][w] = 0;
+    }
+    if constexpr (BITS == 8) {
+        uint4 *o = reinterpret_cast<uint4 *>(codes_out);
+        o[0] = make_uint4(p[0][0], p[0][1], p[1][0], p[1][1]);
+        o[1] = make_uint4(p[2][0], p[2][1], p[3][0], p[3][1]);
+    }
+    if constexpr (BITS == 4)
+        *reinterpret_cast<uint4 *>(codes_out) = make_uint4(p[0][0], p[1][0], p[2][0], p[3][0]);
+    if constexpr (BITS == 2)
+        *reinterpret_cast<uint2 *>(codes_out) = make_uint2(__byte_perm(p[0][0], p[1][0], 0x5410),
+                                                           __byte_perm(p[2][0], p[3][0], 0x5410));
+}
+
+template <int BITS, int C>
+__device__ __forceinline__ void enc_consume_v(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                           int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int gpr = c >> 5;                              // groups per row
+    const int ngroups = nt * gpr;                        // the tile's groups, in stream order
+    const int rot = (tid >> 1) & 3;
+    uint32_t off[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) off[j] = (uint32_t)((j + rot) & 3) * 16u;
+    const size_t g_first = (size_t)tile * kTileTokens * gpr;      // the tile's first group within the plane
+    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec) + g_first;
+    uint8_t *codes = codes_sec + g_first * (4 * BITS);
+    constexpr int U = 2;                                 // groups a thread holds at a time
+    const int iters = (ngroups + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);  // the same for every thread
+    for (int it = 0; it < iters; ++it) {
+        const int g0 = it * kEncGroupThreads * U + tid;
+        uint4 x[U][4];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int g = g0 + k * kEncGroupThreads;
+            if (g < ngroups) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) x[k][j] = *reinterpret_cast<const uint4 *>(st + (size_t)g * 64 + off[j]);
+            }
+        }
+        if (it == iters - 1) enc_release(empty_bar);
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int g = g0 + k * kEncGroupThreads;
+            if (g < ngroups) enc_group_v<BITS>(x[k], rot, meta + g, codes + (size_t)g * (4 * BITS));
+        }
+    }
+}
+
+// One unit of a known level: K or V (or the raw copy), inlined into the caller.
+template <int C, int LEVEL>
+__device__ __forceinline__ void enc_consume_level(const EncUnit &u, const uint8_t *st, int c_rt, int tid,
+                                                  uint64_t *eb)
+{
+    if constexpr (LEVEL == 0) {
+        enc_consume_raw<C>(st, c_rt, tid, eb, u.nt, u.tile, u.codes);
+    } else {
+        constexpr int BITS = 16 >> LEVEL;
+        if (u.kv) enc_consume_v<BITS, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        else if (u.nt == kTileTokens) enc_consume_k<BITS, C>(st, c_rt, tid, eb, u.tile, u.meta, u.codes);
+        else enc_consume_k_short<BITS>(st, C ? C : c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+    }
+}
+// The same as a function of its own: a kernel that has to hold all four levels keeps each level's
+// registers apart this way (inlined side by side they spill).
+template <int C, int LEVEL>
+__device__ __noinline__ void enc_consume_level_call(const EncUnit *u, const uint8_t *st, int c_rt, int tid,
+                                                    uint64_t *eb)
+{
+    enc_consume_level<C, LEVEL>(*u, st, c_rt, tid, eb);
+}
+
+// LEVEL >= 0: every chunk of the launch has this level (checked by the producer); -1: any mix.
+template <int C, int LEVEL>
+__device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st, int c_rt, int tid, uint64_t *eb)
+{
+    if constexpr (LEVEL >= 0) {
+        enc_consume_level<C, LEVEL>(u, st, c_rt, tid, eb);
+    } else {
+        switch (u.bits) {                                // uniform per consumer group
+        case 16: enc_consume_level_call<C, 0>(&u, st, c_rt, tid, eb); break;
+        case 8: enc_consume_level_call<C, 1>(&u, st, c_rt, tid, eb); break;
+        case 4: enc_consume_level_call<C, 2>(&u, st, c_rt, tid, eb); break;
+        default: enc_consume_level_call<C, 3>(&u, st, c_rt, tid, eb); break;
+        }
+    }
+}
+
+// sched: 0 = each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (grid = resident CTAs);
+//        1 = one CTA per tile in the grid, running CTAs pull further tiles through cluster launch control.
+// G consumer groups of 256 threads take the units in turn (unit i goes to group i % G).
+template <int C, int G, int LEVEL>
+__global__ void __launch_bounds__(32 + G * kEncGroupThreads, 1)
+encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
+{
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    __shared__ __align__(8) uint64_t full_bar[kEncStages];
+    __shared__ __align__(8) uint64_t empty_bar[kEncStages];
+    __shared__ EncUnit info[kEncStages];
+    __shared__ int abort_flag;
+    __shared__ __align__(16) uint4 clc_response[2];
+    __shared__ __align__(8) uint64_t clc_bar[2];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kProducerWarp = G * kEncGroupThreads / 32;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kEncStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kEncGroupThreads / 32);
+        }
+        mbar_init(&clc_bar[0], 1);
+        mbar_init(&clc_bar[1], 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kProducerWarp) {
+        // ------------------------------ producer warp ------------------------------
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        uint32_t unit = 0;
+        bool ok = true;
+
+        auto acquire = [&]() -> bool {                   // wait until the unit's stage is free
+            const int s = unit % kEncStages;
+            if (unit < (uint32_t)kEncStages) return true;
+            bool w = true;
+            if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / kEncStages) - 1) & 1, &abort_flag);
+            return __shfl_sync(0xffffffffu, w, 0);
+        };
+
+        auto do_tile = [&](int64_t tile_id) {
+            const int tile = (int)(tile_id % kTilesPerChunk);
+            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int kv = (int)(plane_id & 1);
+            const int layer = (int)((plane_id >> 1) % p.l);
+            const int chunk = p.chunk0 + (int)((plane_id >> 1) / p.l);
+            const int64_t tok0 = (int64_t)chunk * kChunkTokens;
+            const int n_expect = (int)min((int64_t)kChunkTokens, p.N - tok0);
+            kvh_chunk_desc d;
+            if (p.descs) {
+                d = p.descs[chunk];
+            } else {
+                d.stream_off = (uint64_t)chunk * p.full_chunk_bytes;
+                d.level = p.level;
+                d.n_tok = n_expect;
+            }
+            int err = check_desc(d, p.l, p.c, p.capacity);
+            if (err == KVH_OK && d.n_tok != n_expect) err = KVH_ERR_BAD_SHAPE;
+            if (err == KVH_OK && LEVEL >= 0 && d.level != LEVEL) err = KVH_ERR_BAD_LEVEL;
+            if (err != KVH_OK) {
+                if (lane == 0) report(p.status, err);
+                return;
+            }
+            const int n = d.n_tok;
+            const int nt = min(kTileTokens, n - tile * kTileTokens);
+            if (nt <= 0) return;
+            const LayerLayout L = layer_layout(d.level, p.c, n);
+            uint8_t *lay = p.out + d.stream_off + (uint64_t)layer * L.layer_bytes();
+            const uint16_t *src = p.kv + (((int64_t)layer * 2 + kv) * p.N + tok0 + tile * kTileTokens) * p.c;
+            ok = acquire();
+            if (!ok) return;
+            if (lane == 0) {
+                const int s = unit % kEncStages;
+                EncUnit &u = info[s];
+                u.bits = level_bits(d.level); u.kv = kv; u.nt = nt; u.tile = tile;
+                u.last = tile * kTileTokens + nt == n;
+                u.meta_payload = (uint32_t)(kv ? L.vmeta_payload : L.kmeta_payload);
+                u.meta_padded = (uint32_t)(kv ? L.vmeta : L.kmeta);
+                u.codes_payload = (uint32_t)L.codes_payload;
+                u.codes_padded = (uint32_t)L.kcodes;
+                u.meta = lay + L.meta_off(kv);
+                u.codes = lay + L.codes_off(kv);
+                const uint32_t bytes = 2u * (uint32_t)nt * (uint32_t)p.c;       // a multiple of 64
+                mbar_arrive_expect_tx(&full_bar[s], bytes);
+                bulk_load(stage_mem + (size_t)s * kEncStageBytes, src, bytes, &full_bar[s]);
+            }
+            ++unit;
+        };
+
+        int64_t tile_id = blockIdx.x;
+        uint32_t query = 0;                              // answers asked for so far
+        bool asked = false;                              // one answer still outstanding
+        while (ok && tile_id < total_tiles) {
+            if (sched == 1) {                            // ask for the next tile while this one streams
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&clc_bar[query & 1], 16);
+                    clc_try_cancel(&clc_response[query & 1], &clc_bar[query & 1]);
+                }
+                asked = true;
+            }
+            do_tile(tile_id);
+            if (!ok) break;
+            if (sched == 1) {
+                uint32_t got = 0, next = 0, w = 1;
+                if (lane == 0) {
+                    w = mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &abort_flag);
+                    if (w) got = clc_query(&clc_response[query & 1], next);
+                }
+                w = __shfl_sync(0xffffffffu, w, 0);
+                got = __shfl_sync(0xffffffffu, got, 0);
+                next = __shfl_sync(0xffffffffu, next, 0);
+                if (!w) { ok = false; break; }
+                asked = false;
+                ++query;
+                if (!got) break;                         // no CTA left to take over: never ask again
+                tile_id = next;
+            } else {
+                tile_id += gridDim.x;
+            }
+        }
+        for (int g = 0; ok && g < G; ++g) {              // one end marker per consumer group
+            ok = acquire();
+            if (ok) {
+                if (lane == 0) {
+                    info[unit % kEncStages].bits = 0;
+                    mbar_arrive(&full_bar[unit % kEncStages]);
+                }
+                ++unit;
+            }
+        }
+        if (!ok && lane == 0) {
+            report(p.status, KVH_ERR_TIMEOUT);
+            abort_flag = 1;
+        }
+        // Leave only after every copy issued has landed: a normal run has seen them all consumed;
+        // after an abort the last kEncStages units may still be in flight.
+        if (lane == 0) {
+            int never = 0;                               // the drain ignores the abort flag
+            const uint32_t first = unit > (uint32_t)kEncStages ? unit - kEncStages : 0;
+            for (uint32_t w = first; w < unit; ++w)
+                (void)mbar_wait(&full_bar[w % kEncStages], (w / kEncStages) & 1, &never);
+            if (asked) (void)mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &never);
+        }
+    } else {
+        // ------------------------------ consumer warps ------------------------------
+        const int group = warp / (kEncGroupThreads / 32);
+        const int tid = threadIdx.x - group * kEncGroupThreads;
+        for (uint32_t unit = group;; unit += G) {
+            const int s = unit % kEncStages;
+            if (!mbar_wait(&full_bar[s], (unit / kEncStages) & 1, &abort_flag)) {
+                report(p.status, KVH_ERR_TIMEOUT);
+                abort_flag = 1;
+                break;
+            }
+            const EncUnit u = info[s];
+            if (u.bits == 0) break;
+            const uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+            uint64_t *eb = &empty_bar[s];
+            if (u.last && tid < KVH_SECTION_ALIGN) {     // the plane's last tile clears the padding
+                if (u.codes_payload + tid < u.codes_padded) u.codes[u.codes_payload + tid] = 0;
+                if (u.bits < 16 && u.meta_payload + tid < u.meta_padded) u.meta[u.meta_payload + tid] = 0;
+            }
+            enc_dispatch<C, LEVEL>(u, st, p.c, tid, eb);
+        }
+    }
+}
+
+}  // namespace kvh

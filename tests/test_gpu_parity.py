@@ -90,12 +90,13 @@ SHAPES = [
 @pytest.mark.parametrize("l,c,N", SHAPES)
 @pytest.mark.parametrize("level", [0, 1, 2, 3])
 def test_encode_and_decode_match_oracle(kvh, monkeypatch, l, c, N, level, path):
-    # "default" takes the persistent TMA decode kernel where it applies (c <= 1024); "direct"
-    # forces the one-CTA-per-tile kernel on every shape
-    if path == "direct":
-        monkeypatch.setenv("KVH_DECODE_PATH", "direct")
-    else:
-        monkeypatch.delenv("KVH_DECODE_PATH", raising=False)
+    # "default" takes the persistent TMA-fed encode and decode kernels where they apply
+    # (c <= 1024); "direct" forces the one-CTA-per-tile kernels on every shape
+    for var in ("KVH_DECODE_PATH", "KVH_ENCODE_PATH"):
+        if path == "direct":
+            monkeypatch.setenv(var, "direct")
+        else:
+            monkeypatch.delenv(var, raising=False)
     kv = workloads.make_kv(l, N, c, seed=1000 * level + N + c, device="cuda")
     kv_np = to_np16(kv).copy()
     special_values(kv_np, N)
