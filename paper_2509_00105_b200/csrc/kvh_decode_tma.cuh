@@ -59,9 +59,10 @@ template <> struct Pos<8> {
     __device__ static __forceinline__ float prescale(int) { return 1.0f; }
 };
 
-// q_i * 2^pos(i) as a float, for i = 0..7, from the 8 codes of one thread
+// q_i * 2^pos(i) as floats, for i = 0..7, from the 8 codes of one thread: x[k] holds elements 2k and
+// 2k+1 (the subtraction of 2^23 is exact, two elements per instruction)
 template <int BITS>
-__device__ __forceinline__ void spread8(const uint8_t *src, float (&x)[8])
+__device__ __forceinline__ void spread8(const uint8_t *src, f32x2 (&x)[4])
 {
     constexpr uint32_t magic = 0x4b000000u;
     uint32_t m[8];
@@ -91,14 +92,22 @@ __device__ __forceinline__ void spread8(const uint8_t *src, float (&x)[8])
             m[i + 4] = __byte_perm(w.y, magic, 0x7440 + i);
         }
     }
+    const f32x2 bias = f2_from_bits(magic, magic);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] = __fsub_rn(__uint_as_float(m[i]), 8388608.0f);
+    for (int k = 0; k < 4; ++k) x[k] = f2_sub(f2_from_bits(m[2 * k], m[2 * k + 1]), bias);
 }
 
-__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+// bf16_rne of x[k] * sc[k] + lo[k] for the 8 elements, one rounding each
+__device__ __forceinline__ uint4 fma_pack8(const f32x2 (&x)[4], const f32x2 (&sc)[4], const f32x2 (&lo)[4])
 {
-    return make_uint4(pack_bf16x2_rn(f[0], f[1]), pack_bf16x2_rn(f[2], f[3]),
-                      pack_bf16x2_rn(f[4], f[5]), pack_bf16x2_rn(f[6], f[7]));
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        uint32_t a, b;
+        f2_bits(f2_fma(x[k], sc[k], lo[k]), a, b);
+        w[k] = pack_bf16x2_rn(__uint_as_float(a), __uint_as_float(b));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // Rows of a unit are dealt to threads in runs of `rpt` consecutive rows (a power of two, so a run
@@ -149,15 +158,21 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     const int c = C ? C : p.c;
     const RowRun r = row_run<C>(p, u);
     if (r.count == 0) return;
-    float lo[8], sc[8];
+    f32x2 lo[4], sc[4];
     {
         const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * r.cv;
         const uint4 m0 = m[0], m1 = m[1];
         const uint32_t w[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+        float l1[8], s1[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            decode_params<BITS>(w[i], lo[i], sc[i]);
-            sc[i] = __fmul_rn(sc[i], Pos<BITS>::prescale(i));
+            decode_params<BITS>(w[i], l1[i], s1[i]);
+            s1[i] = __fmul_rn(s1[i], Pos<BITS>::prescale(i));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            lo[k] = f2_make(l1[2 * k], l1[2 * k + 1]);
+            sc[k] = f2_make(s1[2 * k], s1[2 * k + 1]);
         }
     }
     const uint32_t row_bytes = (uint32_t)c * BITS / 8;
@@ -165,11 +180,9 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     uint16_t *dst = r.dst;
 #pragma unroll 4
     for (int k = 0; k < r.count; ++k) {
-        float x[8], f[8];
+        f32x2 x[4];
         spread8<BITS>(src, x);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], sc[i], lo[i]);
-        *reinterpret_cast<uint4 *>(dst) = pack8(f);
+        *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
         src += row_bytes;
         dst += c;
     }
@@ -201,14 +214,13 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
             if (kb + j < r.count) {
                 const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
                 const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
-                float s[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) s[i] = __fmul_rn(s0, Pos<BITS>::prescale(i));
-                float x[8], f[8];
+                const f32x2 sa = f2_make(__fmul_rn(s0, Pos<BITS>::prescale(0)), __fmul_rn(s0, Pos<BITS>::prescale(1)));
+                const f32x2 sb = f2_make(__fmul_rn(s0, Pos<BITS>::prescale(2)), __fmul_rn(s0, Pos<BITS>::prescale(3)));
+                const f32x2 ll = f2_make(l1, l1);
+                const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+                f32x2 x[4];
                 spread8<BITS>(src, x);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) f[i] = __fmaf_rn(x[i], s[i & 3], l1);
-                *reinterpret_cast<uint4 *>(dst) = pack8(f);
+                *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
                 src += row_bytes;
                 dst += c;
             }

@@ -115,6 +115,40 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float a, float b)
     return r;
 }
 
+// ---- two binary32 values in one 64-bit register -----------------------------------------------
+
+typedef unsigned long long f32x2;
+
+__device__ __forceinline__ f32x2 f2_from_bits(uint32_t a, uint32_t b)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_make(float a, float b) { return f2_from_bits(__float_as_uint(a), __float_as_uint(b)); }
+__device__ __forceinline__ void f2_bits(f32x2 v, uint32_t &a, uint32_t &b)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 f2_sub(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_mul(f32x2 a, f32x2 b)
+{
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 f2_fma(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 // Order-preserving 16-bit keys for two packed bf16: numeric order, -0 below +0.
 __device__ __forceinline__ uint32_t order_keys2(uint32_t pair)
 {
