@@ -44,7 +44,9 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one decode launch relative to its algorithmic bytes, from the ncu capture
 # summarised in profiles/decode_tma_kernel_llama3-70b.md (dram__bytes_read + dram__bytes_write
 # on a 4096-token slice of the same workload; traffic grows in proportion to the tokens).
-DRAM_TRAFFIC_RATIO = {0: 0.981, 1: 0.973, 2: 0.967, 3: 0.963}
+DRAM_TRAFFIC_RATIO = {0: 0.981, 1: 0.973, 2: 0.968, 3: 0.965}
+# the same for one encode launch (profiles/encode_tma_kernel_llama3-70b.md)
+ENCODE_DRAM_TRAFFIC_RATIO = {0: 0.979, 1: 0.978, 2: 0.987, 3: 0.991}
 
 
 def measured_peak() -> tuple[float, str]:
@@ -178,6 +180,26 @@ def run_reference(args, shape: workloads.Shape):
 # the CUDA library
 # ------------------------------------------------------------------------------------------
 
+def rank_seed(rank: int) -> int:
+    """Every rank encodes and loads a context of its own (weak scaling: replicas, no exchange)."""
+    return 3000 + rank
+
+
+def max_over_ranks(values: list[float], device, world: int) -> list[float]:
+    """Element-wise maximum of per-rank timings: the job is as slow as its slowest rank."""
+    if world == 1:
+        return list(values)
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_gbps(world: int, bytes_per_rank: float, ms: float) -> float:
+    """Aggregate throughput of `world` ranks that each moved bytes_per_rank in (at most) ms."""
+    return world * bytes_per_rank / ms / 1e6
+
+
 def run_ours(args, shape: workloads.Shape):
     import torch.distributed as dist
     import paper_2509_00105_b200 as kvh
@@ -195,9 +217,9 @@ def run_ours(args, shape: workloads.Shape):
     elements = l * 2 * N * c
     n_chunks = workloads.n_chunks(N)
     n_pages = workloads.n_pages(N)
-    kv = workloads.make_kv(l, N, c, seed=3000 + rank, device=dev)      # every rank its own context
+    kv = workloads.make_kv(l, N, c, seed=rank_seed(rank), device=dev)   # every rank its own context
     pool = kvh.Pool.allocate(l, n_pages, c, device=dev)
-    table = workloads.shuffled_page_table(n_pages, n_pages, seed=3000 + rank).to(dev)
+    table = workloads.shuffled_page_table(n_pages, n_pages, seed=rank_seed(rank)).to(dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     plans = {}
     for level in LEVELS:
@@ -242,11 +264,7 @@ def run_ours(args, shape: workloads.Shape):
     total_ms = t_start.elapsed_time(t_end)
     enc_ms = {lv: sum(e[lv][0].elapsed_time(e[lv][1]) for e in ev) / args.steps for lv in LEVELS}
     dec_ms = {lv: sum(e[lv][1].elapsed_time(e[lv][2]) for e in ev) / args.steps for lv in LEVELS}
-    times = torch.tensor([total_ms] + [enc_ms[lv] for lv in LEVELS] + [dec_ms[lv] for lv in LEVELS],
-                         dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    times = times.tolist()
+    times = max_over_ranks([total_ms] + [enc_ms[lv] for lv in LEVELS] + [dec_ms[lv] for lv in LEVELS], dev, world)
     total_ms = times[0]
     enc_ms = dict(zip(LEVELS, times[1:5]))
     dec_ms = dict(zip(LEVELS, times[5:9]))
@@ -276,19 +294,15 @@ def run_ours(args, shape: workloads.Shape):
                     if it > 0:
                         store_ms[level] += a.elapsed_time(b) / k_e2e
                         load_ms[level] += b.elapsed_time(d) / k_e2e
-        t = torch.tensor([load_ms[lv] for lv in LEVELS] + [store_ms[lv] for lv in LEVELS], dtype=torch.float64,
-                         device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t = t.tolist()
+        t = max_over_ranks([load_ms[lv] for lv in LEVELS] + [store_ms[lv] for lv in LEVELS], dev, world)
         load_ms, store_ms = dict(zip(LEVELS, t[:4])), dict(zip(LEVELS, t[4:]))
         stream_total = sum(plans[lv][2] for lv in LEVELS)
-        e2e = {"value": world * len(LEVELS) * 2 * elements / sum(load_ms.values()) / 1e6, "unit": UNIT,
+        e2e = {"value": whole_job_gbps(world, len(LEVELS) * 2 * elements, sum(load_ms.values())), "unit": UNIT,
                "h2d_bytes_per_step": stream_total, "d2h_bytes_per_step": stream_total + 4 * 2 * len(LEVELS),
                "steps": k_e2e, "what": "kvh_load_host: pinned host streams -> HBM -> pages, status read back",
                "load_ms_per_level": [round(load_ms[lv], 3) for lv in LEVELS],
                "store_ms_per_level": [round(store_ms[lv], 3) for lv in LEVELS],
-               "store_gbps_bf16_in": world * len(LEVELS) * 2 * elements / sum(store_ms.values()) / 1e6}
+               "store_gbps_bf16_in": whole_job_gbps(world, len(LEVELS) * 2 * elements, sum(store_ms.values()))}
         del host
 
     if rank != 0:
@@ -314,7 +328,7 @@ def run_ours(args, shape: workloads.Shape):
     if all(r is not None for r in ratios):
         traffic = sum(r * algorithmic_bytes(lv, elements, plans[lv][2]) for r, lv in zip(ratios, LEVELS)) / len(LEVELS)
     out = {
-        "metric": METRIC, "value": world * len(LEVELS) * 2 * elements / dec_total_ms / 1e6, "unit": UNIT,
+        "metric": METRIC, "value": whole_job_gbps(world, len(LEVELS) * 2 * elements, dec_total_ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": shape.name, "n_layers": l, "n_channels": c, "n_tokens": N, "chunk_tokens": 256,
@@ -327,6 +341,12 @@ def run_ours(args, shape: workloads.Shape):
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                      "frac_of_8TBs_datasheet": achieved / 8000.0,
                      "per_launch": "mean over the 4 launches of a step (one per level): stream bytes + 2 B/element"},
+        "roofline_encode": {"bound": "hbm", "kernel": "encode_tma_kernel", "achieved": alg_total / sum(enc_ms.values()) / 1e6,
+                            "peak": peak, "unit": "GB/s", "frac": alg_total / sum(enc_ms.values()) / 1e6 / peak,
+                            "traffic": sum(ENCODE_DRAM_TRAFFIC_RATIO[lv] * algorithmic_bytes(lv, elements, plans[lv][2])
+                                           for lv in LEVELS) / len(LEVELS),
+                            "peak_kind": f"of {peak_kind}",
+                            "per_launch": "mean over the 4 launches of a step: 2 B/element + stream bytes"},
         "gpu_launches": args.steps * 2 * len(LEVELS),
         "clocks": clocks,
     }
