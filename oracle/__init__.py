@@ -220,3 +220,62 @@ def decode_context(stream: np.ndarray, offsets, ntoks, levels, l: int, c: int,
                                 page_table[i * pages_per_chunk:], pool, layer_stride,
                                 kv_stride, page_stride, num_pages, page_tokens)
     return skipped
+
+
+# ---- token dropping (the paper's second compression method) -----------------
+#
+# The paper names token dropping beside quantisation (Introduction: texts that matter only "at
+# the beginning and the end" suit it) and cites the attention-sink method for it: the first few
+# tokens and a window of the most recent ones are kept, the middle is dropped.  The kept tokens
+# are stored compacted, in order, as an ordinary context of n_kept tokens at any level; the rate
+# of the method is n_kept / N.  The definition is therefore "encode the compacted tensor".
+
+def keep_sinks_and_recent(N: int, n_sink: int, n_recent: int) -> list[tuple[int, int]]:
+    """Kept runs (first token, count) when the first n_sink and the last n_recent tokens of an
+    N-token context survive; everything if the two windows meet."""
+    if N <= 0 or n_sink < 0 or n_recent < 0:
+        raise ValueError("invalid arguments")
+    if n_sink + n_recent >= N:
+        return [(0, N)]
+    runs = []
+    if n_sink:
+        runs.append((0, n_sink))
+    if n_recent:
+        runs.append((N - n_recent, n_recent))
+    return runs
+
+
+def compact_tokens(kv: np.ndarray, runs) -> np.ndarray:
+    """kv[l][2][N][c] restricted to the kept runs, in order: [l][2][n_kept][c]."""
+    prev_end = 0
+    for first, count in runs:
+        if count <= 0 or first < prev_end or first + count > kv.shape[2]:
+            raise ValueError("runs must be ascending, disjoint, non-empty and inside the context")
+        prev_end = first + count
+    return np.ascontiguousarray(np.concatenate([kv[:, :, f:f + n, :] for f, n in runs], axis=2))
+
+
+def encode_kept(kv: np.ndarray, runs, levels) -> tuple[np.ndarray, list[int]]:
+    """Stored form of a context after token dropping: the chunks of the compacted tensor."""
+    return encode_context(compact_tokens(kv, runs), levels)
+
+
+# ---- transcoding a stored chunk to a lower quality level ---------------------
+#
+# The policy's marginal-utility step may "compress furthermore" an entry that is already stored.
+# What is stored is all there is to compress, so the result is defined as the encoding, at the
+# new level, of the values the stored chunk decodes to.
+
+def decode_chunk_values(chunk: np.ndarray, level: int, l: int, c: int, n: int) -> np.ndarray:
+    """The bf16 values a stored chunk decodes to, [l][2][n][c] (uint16 bit patterns)."""
+    npg = (n + 15) // 16
+    pool = np.zeros(l * 2 * npg * 16 * c, dtype=np.uint16)
+    skipped = decode_chunk(chunk, level, l, c, n, np.arange(npg, dtype=np.int32), pool,
+                           2 * npg * 16 * c, npg * 16 * c, 16 * c, npg)
+    assert skipped == 0
+    return np.ascontiguousarray(pool.reshape(l, 2, npg * 16, c)[:, :, :n, :])
+
+
+def transcode_chunk(chunk: np.ndarray, level_in: int, level_out: int, l: int, c: int, n: int) -> np.ndarray:
+    """encode(level_out) of decode(level_in) of a stored chunk."""
+    return encode_chunk(decode_chunk_values(chunk, level_in, l, c, n), 0, n, level_out)

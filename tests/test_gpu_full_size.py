@@ -15,16 +15,16 @@ from test_gpu_parity import SENTINEL, kvh, to_np16  # noqa: F401
 pytestmark = pytest.mark.gpu
 
 
-def check_sampled_chunks(kvh, kv, level_of_chunk, sample, streams, descs, table, pool, spare_pages):
-    """kv: [l][2][N][c] on the GPU; streams/descs: what the GPU encoded; pool: decoded into."""
-    l, _, N, c = kv.shape
+def check_sampled_chunks(kvh, chunk_src, N, level_of_chunk, sample, streams, descs, table, pool, spare_pages):
+    """chunk_src(i): the source tokens of chunk i, [l][2][n][c] on the GPU; streams/descs: what the
+    GPU encoded; pool: what it decoded into."""
     ptable = table.cpu().numpy()
 
     def one(i):
-        tok0 = 256 * i
-        n = min(256, N - tok0)
+        src = to_np16(chunk_src(i))
+        l, _, n, c = src.shape
+        assert n == min(256, N - 256 * i)
         level = level_of_chunk(i)
-        src = to_np16(kv[:, :, tok0:tok0 + n, :])
         want = oracle.encode_chunk(np.ascontiguousarray(src), 0, n, level)
         off = int(descs["stream_off"][i])
         got = streams[off:off + want.size].cpu().numpy()
@@ -61,7 +61,8 @@ def run_context(kvh, shape, seed, levels, sample):
         assert used == total
         kvh.decode_batch(streams, kvh.descs_to_tensor(descs, "cuda"), len(descs), table, pool, status)
         assert status.item() == 0
-        check_sampled_chunks(kvh, kv, lambda i: level, sample, streams, descs, table, pool, perm[n_pages:].tolist())
+        check_sampled_chunks(kvh, lambda i: kv[:, :, 256 * i:min(N, 256 * i + 256)], N, lambda i: level, sample, streams,
+                             descs, table, pool, perm[n_pages:].tolist())
         del streams
 
 
@@ -83,16 +84,25 @@ def test_llama8b_128k_offsets_beyond_32_bits(kvh):
 
 
 def test_batched_mixed_level_load_at_scale(kvh):
-    """64 contexts, lengths log-uniform in [2K, 32K] with partial last chunks, a random level per
-    chunk, one shared pool behind one shuffled page table, ONE decode launch.  Eight layers
-    instead of 32 keep the pool at ~23 GB; the launch geometry per layer is the benchmark's."""
-    l, c = 8, 1024
+    """The batched mixed-level workload at its full size: 64 contexts of the 8B shape (32 layers),
+    lengths log-uniform in [2K, 32K] with partial last chunks, a random level per chunk, one shared
+    pool (~93 GB) behind one shuffled page table, ONE decode launch over ~2,800 chunks (~48 GB of
+    streams).  On a GPU with less free memory the layer count is reduced to what fits; the launch
+    geometry per layer stays the benchmark's."""
+    c = 1024
     lengths = workloads.context_lengths(workloads.BATCH_N_CONTEXTS, workloads.BATCH_MIN_TOKENS,
                                         workloads.BATCH_MAX_TOKENS, seed=3000)
     assert len(lengths) == 64 and min(lengths) >= 2048 and max(lengths) <= 32768
     assert any(n % 256 for n in lengths)
     total_pages = sum(workloads.n_pages(n) for n in lengths)
     num_pages = total_pages + 100
+    all_levels = [workloads.chunk_levels(workloads.n_chunks(N), 4, seed=3100 + i) for i, N in enumerate(lengths)]
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    per_layer = 2 * num_pages * 16 * c * 2                                   # pool
+    per_layer += sum(kvh.plan_chunks(1, c, N, lv)[1] for N, lv in zip(lengths, all_levels))   # streams
+    per_layer += 2 * 2 * max(lengths) * c * 2                                # one context's KV and slack
+    l = int(max(1, min(32, (free - (12 << 30)) // per_layer)))
     perm = workloads.shuffled_page_table(num_pages, num_pages, seed=3001)
     table = perm[:total_pages].cuda()
     pool = kvh.Pool.allocate(l, num_pages, c)
@@ -101,13 +111,12 @@ def test_batched_mixed_level_load_at_scale(kvh):
 
     plans, total_bytes, pt_base = [], 0, 0
     for i, N in enumerate(lengths):
-        levels = workloads.chunk_levels(workloads.n_chunks(N), 4, seed=3100 + i)
-        descs, size = kvh.plan_chunks(l, c, N, levels, stream_base=total_bytes, pt_base=pt_base)
-        plans.append((N, levels, descs))
+        descs, size = kvh.plan_chunks(l, c, N, all_levels[i], stream_base=total_bytes, pt_base=pt_base)
+        plans.append((N, all_levels[i], descs))
         total_bytes += size
         pt_base += workloads.n_pages(N)
     blob = torch.empty(total_bytes, dtype=torch.uint8, device="cuda")
-    kept = {}
+    kept = {}                                          # (context, chunk) -> the chunk's source tokens
     for i, (N, levels, descs) in enumerate(plans):
         kv = workloads.make_kv(l, N, c, seed=3200 + i, device="cuda")
         local = descs.copy()
@@ -116,12 +125,15 @@ def test_batched_mixed_level_load_at_scale(kvh):
         size = int(local["stream_off"][-1]) + kvh.level_bytes(int(local["level"][-1]), l, c, int(local["n_tok"][-1]))
         kvh.encode_chunks(kv, kvh.descs_to_tensor(local, "cuda"), len(local), blob[base:base + size], status)
         if i in (0, 17, 63):
-            kept[i] = kv
+            last = len(levels) - 1
+            for j in (0, last // 2, last):
+                kept[(i, j)] = kv[:, :, 256 * j:min(N, 256 * j + 256)].clone()
+        del kv
     all_descs = np.concatenate([d for _, _, d in plans])
     kvh.decode_batch(blob, kvh.descs_to_tensor(all_descs, "cuda"), len(all_descs), table, pool, status)
     assert status.item() == 0
-    for i, kv in kept.items():
+    for i in (0, 17, 63):
         N, levels, descs = plans[i]
-        last = len(levels) - 1
-        check_sampled_chunks(kvh, kv, lambda j: levels[j], [0, last // 2, last], blob, descs, table, pool,
+        sample = sorted(j for (ci, j) in kept if ci == i)
+        check_sampled_chunks(kvh, lambda j: kept[(i, j)], N, lambda j: levels[j], sample, blob, descs, table, pool,
                              perm[total_pages:].tolist() if i == 0 else None)

@@ -467,3 +467,106 @@ def test_context_plan_offsets():
                        oracle.level_bytes(3, l, c, 256) + oracle.level_bytes(0, l, c, 256),
                        oracle.level_bytes(3, l, c, 256) + oracle.level_bytes(0, l, c, 256) + oracle.level_bytes(2, l, c, 37)]
     assert all(o % 128 == 0 for o in offsets)
+
+
+# ---- token dropping and transcoding (composed from the steps pinned above) -------------------
+
+def _rand_kv(l, N, c, seed):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((l, 2, N, c)).astype(np.float32)
+    return np.ascontiguousarray((x.view(np.uint32) >> 16).astype(np.uint16))
+
+
+def test_kept_runs_of_sinks_and_recent_window():
+    assert oracle.keep_sinks_and_recent(1000, 4, 252) == [(0, 4), (748, 252)]
+    assert oracle.keep_sinks_and_recent(1000, 0, 10) == [(990, 10)]
+    assert oracle.keep_sinks_and_recent(1000, 10, 0) == [(0, 10)]
+    assert oracle.keep_sinks_and_recent(100, 60, 40) == [(0, 100)]        # windows meet: nothing dropped
+    assert oracle.keep_sinks_and_recent(100, 80, 40) == [(0, 100)]
+    with pytest.raises(ValueError):
+        oracle.keep_sinks_and_recent(0, 1, 1)
+
+
+def test_compaction_keeps_exactly_the_kept_tokens_in_order():
+    """Token by token: compacted position j holds the j-th kept source token, nothing else."""
+    kv = _rand_kv(2, 700, 32, 1)
+    runs = [(0, 4), (300, 37), (650, 50)]
+    got = oracle.compact_tokens(kv, runs)
+    kept = [t for f, n in runs for t in range(f, f + n)]
+    assert got.shape == (2, 2, len(kept), 32)
+    for j, t in enumerate(kept):
+        assert np.array_equal(got[:, :, j], kv[:, :, t])
+    for bad in ([(5, 3), (6, 2)], [(10, 0)], [(690, 20)], [(20, 5), (0, 5)]):
+        with pytest.raises(ValueError):
+            oracle.compact_tokens(kv, bad)
+
+
+def test_dropping_at_level_0_stores_the_kept_tokens_and_nothing_else():
+    l, N, c = 2, 900, 64
+    kv = _rand_kv(l, N, c, 2)
+    runs = oracle.keep_sinks_and_recent(N, 4, 380)
+    stream, offsets = oracle.encode_kept(kv, runs, 0)
+    n_kept = 384
+    assert len(offsets) == 3 and offsets[-1] == l * 2 * n_kept * c * 2     # size = rate x full size
+    assert offsets[-1] * N == oracle.encode_context(kv, 0)[0].size * n_kept
+    vals = np.concatenate([oracle.decode_chunk_values(stream[offsets[i]:offsets[i + 1]], 0, l, c, n)
+                           for i, n in enumerate((256, 128))], axis=2)
+    assert np.array_equal(vals[:, :, :4], kv[:, :, :4])
+    assert np.array_equal(vals[:, :, 4:], kv[:, :, N - 380:])
+
+
+def test_dropping_then_quantising_groups_the_compacted_tokens():
+    """K groups run over 32 consecutive *kept* tokens: a group that spans the seam between the
+    sink and the recent window takes its range from both sides."""
+    l, N, c = 1, 600, 32
+    kv = _rand_kv(l, N, c, 3)
+    kv[0, 0, 0:4, 0] = 0x4120          # 10.0 in the sinks, channel 0
+    kv[0, 0, 400:, 0] = 0xC120         # -10.0 in the recent window
+    runs = oracle.keep_sinks_and_recent(N, 4, 200)
+    stream, _ = oracle.encode_kept(kv, runs, 3)
+    meta0 = int(stream[:4].view(np.uint32)[0])           # K metadata word of channel 0, first group
+    assert meta0 == (0xC120 | (0x4120 << 16))
+    same = oracle.encode_context(oracle.compact_tokens(kv, runs), 3)[0]
+    assert np.array_equal(stream, same)
+
+
+@pytest.mark.parametrize("level_out", [1, 2, 3])
+def test_transcoding_from_full_quality_is_encoding(level_out):
+    l, c, n = 2, 64, 77
+    kv = _rand_kv(l, n, c, 4)
+    raw = oracle.encode_chunk(kv, 0, n, 0)
+    assert np.array_equal(oracle.decode_chunk_values(raw, 0, l, c, n), kv)
+    assert np.array_equal(oracle.transcode_chunk(raw, 0, level_out, l, c, n), oracle.encode_chunk(kv, 0, n, level_out))
+
+
+@pytest.mark.parametrize("level_in,level_out", [(1, 2), (1, 3), (2, 3), (2, 2), (3, 1)])
+def test_transcoding_against_the_brute_force_path(level_in, level_out):
+    """Byte for byte against the exact-arithmetic implementation, composed the same way."""
+    l, c, n = 1, 32, 45
+    kv = _rand_kv(l, n, c, 5 + level_in)
+    s = oracle.encode_chunk(kv, 0, n, level_in)
+    got = oracle.transcode_chunk(s, level_in, level_out, l, c, n)
+    vals = naive.decode_chunk(bytes(s), level_in, l, c, n)
+    want = naive.encode_chunk(vals, l, c, 0, n, level_out)
+    assert got.size == oracle.level_bytes(level_out, l, c, n)
+    assert bytes(got) == want
+
+
+def test_transcoding_error_and_range_properties():
+    """A transcoded group keeps its minimum exactly, never widens its range, and its values stay
+    within half a step of the new level plus half a step of the old one (plus bf16 rounding)."""
+    l, c, n = 1, 64, 256
+    kv = _rand_kv(l, n, c, 9)
+    x = (kv.astype(np.uint32) << 16).view(np.float32)
+    s1 = oracle.encode_chunk(kv, 0, n, 1)
+    s3 = oracle.transcode_chunk(s1, 1, 3, l, c, n)
+    v1 = (oracle.decode_chunk_values(s1, 1, l, c, n).astype(np.uint32) << 16).view(np.float32)
+    v3 = (oracle.decode_chunk_values(s3, 3, l, c, n).astype(np.uint32) << 16).view(np.float32)
+    k = x[0, 0].reshape(8, 32, c)                        # K groups: [group][token][channel]
+    r = k.max(1) - k.min(1)
+    k3 = v3[0, 0].reshape(8, 32, c)
+    assert np.array_equal(k3.min(1), k.min(1))           # min -> code 0 -> min at both levels
+    assert np.all(k3.max(1) <= k.max(1) + 1e-6)
+    bound = r[:, None, :] * (0.5 / 255 + 0.5 / 3) + 2.0 ** -7 * np.abs(k).max(1)[:, None, :]
+    assert np.all(np.abs(k3 - k) <= bound)
+    assert np.abs(v3 - x).mean() > np.abs(v1 - x).mean()  # and it is the coarser of the two
