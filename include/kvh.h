@@ -134,6 +134,35 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
                              void *out, uint64_t out_capacity,
                              int32_t *dev_status, void *stream);
 
+/* Token dropping, the paper's second compression method (Introduction: contexts that matter "at
+ * the beginning and the end"; the method cited keeps the first tokens, the attention sinks, and a
+ * window of the most recent ones).  A kept run is a range of consecutive source tokens; the kept
+ * tokens of all runs, in order, form the sequence that is stored, at any level, exactly as
+ * kvh_encode_chunks would store a context of n_kept tokens.  On a hit the chunks decode into
+ * consecutive page slots like any other context, so the engine sees the compacted cache. */
+#define KVH_MAX_KEPT_RUNS 8
+typedef struct {
+    int64_t first;         /* first source token of the run */
+    int64_t count;         /* tokens in the run, > 0 */
+} kvh_token_run;
+
+/* Runs kept when the first n_sink and the last n_recent tokens of an n_tokens context survive:
+ * one or two runs, or the single run [0, n_tokens) when the windows meet.  runs_out [host, room
+ * for 2]; *n_runs, *n_kept [host].  Pure host arithmetic. */
+kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n_recent,
+                                     kvh_token_run *runs_out, int *n_runs, int64_t *n_kept);
+
+/* Encode the kept tokens of a context.  kv [device] as for kvh_encode ([n_layers][2][n_tokens]
+ * [n_channels]).  runs [host, n_runs <= KVH_MAX_KEPT_RUNS]: ascending, disjoint, inside the
+ * context.  descs [device, n_chunks = ceil(n_kept / 256)] describe the chunks of the compacted
+ * sequence (lay them out with kvh_plan_chunks for n_kept tokens); everything else as for
+ * kvh_encode_chunks.  n_channels must not exceed 1024 (KVH_ERR_BAD_SHAPE otherwise). */
+kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                           const kvh_token_run *runs, int n_runs,
+                           const kvh_chunk_desc *descs, int n_chunks,
+                           void *out, uint64_t out_capacity,
+                           int32_t *dev_status, void *stream);
+
 /* Decode one stored chunk (cache hit) into the pool.  chunk [device, 128-byte
  * aligned]: the chunk's stream.  page_ids [device]: ceil(n_tok/page_tokens)
  * page ids; token t goes to page page_ids[t / page_tokens], slot

@@ -78,6 +78,10 @@ def lib() -> ctypes.CDLL:
                                     u64, vp, vp]
         L.kvh_store_host.restype = i32
         L.kvh_store_host.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, u64, vp, vp, vp, u64, vp, vp]
+        L.kvh_keep_sinks_and_recent.restype = i32
+        L.kvh_keep_sinks_and_recent.argtypes = [i64, i64, i64, vp, ip, ctypes.POINTER(i64)]
+        L.kvh_encode_kept.restype = i32
+        L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, vp, u64, vp, vp]
         L.kvh_load_host_static.restype = i32
         L.kvh_load_host_static.argtypes = [vp, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp, u64, vp, vp]
         _lib = L
@@ -269,3 +273,27 @@ def load_host_static(host_streams: torch.Tensor, descs: np.ndarray, descs_dev: t
                                       page_table.data_ptr(), page_table.numel(), ctypes.byref(pool.struct),
                                       _ptr(dev_status), _ptr(host_status), slice_bytes, copy_stream.cuda_stream,
                                       _stream()), "kvh_load_host_static")
+
+
+RUN_DTYPE = np.dtype([("first", "<i8"), ("count", "<i8")])
+
+
+def keep_sinks_and_recent(n_tokens: int, n_sink: int, n_recent: int) -> tuple[np.ndarray, int]:
+    """Kept runs (array of RUN_DTYPE) and the number of kept tokens when the first n_sink and the
+    last n_recent tokens of a context survive."""
+    runs = np.zeros(2, dtype=RUN_DTYPE)
+    n, kept = ctypes.c_int(), ctypes.c_int64()
+    _check(lib().kvh_keep_sinks_and_recent(n_tokens, n_sink, n_recent, runs.ctypes.data, ctypes.byref(n),
+                                           ctypes.byref(kept)), "kvh_keep_sinks_and_recent")
+    return runs[:n.value].copy(), kept.value
+
+
+def encode_kept(kv: torch.Tensor, runs, descs_dev: torch.Tensor, n_chunks: int, out: torch.Tensor,
+                dev_status: torch.Tensor | None = None) -> None:
+    """Token dropping: encode only the kept runs of a context, compacted; descs_dev lays out the
+    chunks of the kept sequence (plan_chunks for n_kept tokens)."""
+    l, N, c = _check_kv(kv)
+    r = np.ascontiguousarray(np.asarray(runs, dtype=RUN_DTYPE) if not isinstance(runs, np.ndarray) else runs)
+    assert r.dtype == RUN_DTYPE
+    _check(lib().kvh_encode_kept(kv.data_ptr(), l, N, c, r.ctypes.data, len(r), descs_dev.data_ptr(), n_chunks,
+                                 out.data_ptr(), out.numel(), _ptr(dev_status), _stream()), "kvh_encode_kept")

@@ -110,7 +110,7 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream)
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const char *force = getenv("KVH_ENCODE_PATH");
-    if (p.c <= kEncMaxChannels && !(force && strcmp(force, "direct") == 0)) {
+    if (p.c <= kEncMaxChannels && (p.n_runs > 0 || !(force && strcmp(force, "direct") == 0))) {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -227,7 +227,7 @@ kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_chan
     const int64_t n_chunks = (n_tokens + kChunkTokens - 1) / kChunkTokens;
     EncodeParams p{};
     p.kv = static_cast<const uint16_t *>(kv);
-    p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+    p.l = n_layers; p.c = n_channels; p.N = n_tokens; p.src_N = n_tokens;
     p.descs = nullptr;
     p.level = level;
     p.full_chunk_bytes = chunk_bytes(level, n_layers, n_channels, kChunkTokens);
@@ -248,7 +248,58 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
     if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
     EncodeParams p{};
     p.kv = static_cast<const uint16_t *>(kv);
-    p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+    p.l = n_layers; p.c = n_channels; p.N = n_tokens; p.src_N = n_tokens;
+    p.descs = descs;
+    p.out = static_cast<uint8_t *>(out);
+    p.capacity = out_capacity;
+    p.status = dev_status;
+    return launch_encode(p, n_chunks, stream);
+}
+
+kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n_recent,
+                                     kvh_token_run *runs_out, int *n_runs, int64_t *n_kept)
+{
+    if (!runs_out || !n_runs || n_tokens <= 0 || n_sink < 0 || n_recent < 0) return KVH_ERR_INVALID_ARG;
+    int n = 0;
+    if (n_sink >= n_tokens || n_recent >= n_tokens - n_sink) {      // the windows meet: nothing is dropped
+        runs_out[n++] = kvh_token_run{0, n_tokens};
+    } else {
+        if (n_sink > 0) runs_out[n++] = kvh_token_run{0, n_sink};
+        if (n_recent > 0) runs_out[n++] = kvh_token_run{n_tokens - n_recent, n_recent};
+    }
+    *n_runs = n;
+    if (n_kept) {
+        *n_kept = 0;
+        for (int r = 0; r < n; ++r) *n_kept += runs_out[r].count;
+    }
+    return KVH_OK;
+}
+
+kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
+                           const kvh_token_run *runs, int n_runs, const kvh_chunk_desc *descs, int n_chunks,
+                           void *out, uint64_t out_capacity, int32_t *dev_status, void *stream)
+{
+    if (!kv || !out || !descs || !runs || n_tokens <= 0 || n_runs <= 0 || n_runs > kMaxKeptRuns)
+        return KVH_ERR_INVALID_ARG;
+    const kvh_status s = check_shape(0, n_layers, n_channels);
+    if (s != KVH_OK) return s;
+    if (n_channels > kEncMaxChannels) return KVH_ERR_BAD_SHAPE;       // the gather is the TMA kernel's
+    if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
+    EncodeParams p{};
+    int64_t end = 0, kept = 0;
+    for (int r = 0; r < n_runs; ++r) {
+        if (runs[r].count <= 0 || runs[r].first < end || runs[r].first > n_tokens - runs[r].count)
+            return KVH_ERR_INVALID_ARG;
+        p.run_first[r] = runs[r].first;
+        p.run_pos[r] = kept;
+        end = runs[r].first + runs[r].count;
+        kept += runs[r].count;
+    }
+    p.run_pos[n_runs] = kept;
+    p.n_runs = n_runs;
+    if ((int64_t)n_chunks != (kept + kChunkTokens - 1) / kChunkTokens) return KVH_ERR_BAD_SHAPE;
+    p.kv = static_cast<const uint16_t *>(kv);
+    p.l = n_layers; p.c = n_channels; p.N = kept; p.src_N = n_tokens;
     p.descs = descs;
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
@@ -408,7 +459,7 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
         const Slice s = next_slice(descs_host, n_chunks, i, n_layers, n_channels, slice_bytes);
         EncodeParams p{};
         p.kv = static_cast<const uint16_t *>(kv);
-        p.l = n_layers; p.c = n_channels; p.N = n_tokens;
+        p.l = n_layers; p.c = n_channels; p.N = n_tokens; p.src_N = n_tokens;
         p.descs = descs_dev;
         p.chunk0 = s.first;
         p.out = static_cast<uint8_t *>(dev_staging);

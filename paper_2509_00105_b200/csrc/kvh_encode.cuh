@@ -20,10 +20,19 @@
 
 namespace kvh {
 
+constexpr int kMaxKeptRuns = KVH_MAX_KEPT_RUNS;
+
 struct EncodeParams {
-    const uint16_t *kv;            // [l][2][N][c]
+    const uint16_t *kv;            // [l][2][src_N][c]
     int32_t l, c;
-    int64_t N;
+    int64_t N;                     // tokens that get encoded (the kept ones when runs are given)
+    int64_t src_N;                 // tokens per plane of kv
+    // Token dropping: n_runs > 0 keeps run r = source tokens [run_first[r], run_first[r] + run_pos[r+1]
+    // - run_pos[r]) and stores them compacted, so that kept token j of run r is token run_pos[r] + j
+    // of the encoded sequence.  n_runs == 0: the encoded sequence is the source itself.
+    int32_t n_runs;
+    int64_t run_first[kMaxKeptRuns];
+    int64_t run_pos[kMaxKeptRuns + 1];
     const kvh_chunk_desc *descs;   // device array indexed by chunk, or nullptr for one level throughout
     int32_t chunk0;                // first chunk this launch covers
     int32_t level;                 // used when descs == nullptr
@@ -303,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams 
     uint8_t *lay = p.out + d.stream_off + (uint64_t)layer * L.layer_bytes();
     uint8_t *meta = lay + L.meta_off(kv);
     uint8_t *codes = lay + L.codes_off(kv);
-    const uint16_t *src = p.kv + (((int64_t)layer * 2 + kv) * p.N + tok0 + tile * kTileTokens) * p.c;
+    const uint16_t *src = p.kv + (((int64_t)layer * 2 + kv) * p.src_N + tok0 + tile * kTileTokens) * p.c;
 
     if (tile * kTileTokens + nt == n) {                   // the plane's last tile clears the padding
         zero_pad(codes, L.codes_payload, L.kcodes);

@@ -435,7 +435,8 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
             if (nt <= 0) return;
             const LayerLayout L = layer_layout(d.level, p.c, n);
             uint8_t *lay = p.out + d.stream_off + (uint64_t)layer * L.layer_bytes();
-            const uint16_t *src = p.kv + (((int64_t)layer * 2 + kv) * p.N + tok0 + tile * kTileTokens) * p.c;
+            const uint16_t *plane = p.kv + ((int64_t)layer * 2 + kv) * p.src_N * p.c;
+            const int64_t j0 = tok0 + tile * kTileTokens;        // the tile's first token in the encoded sequence
             ok = acquire();
             if (!ok) return;
             if (lane == 0) {
@@ -449,9 +450,21 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
                 u.codes_padded = (uint32_t)L.kcodes;
                 u.meta = lay + L.meta_off(kv);
                 u.codes = lay + L.codes_off(kv);
-                const uint32_t bytes = 2u * (uint32_t)nt * (uint32_t)p.c;       // a multiple of 64
-                mbar_arrive_expect_tx(&full_bar[s], bytes);
-                bulk_load(stage_mem + (size_t)s * kEncStageBytes, src, bytes, &full_bar[s]);
+                const uint32_t row_bytes = 2u * (uint32_t)p.c;                  // a multiple of 64
+                uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+                mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nt * row_bytes);
+                if (p.n_runs == 0) {
+                    bulk_load(st, plane + j0 * p.c, (uint32_t)nt * row_bytes, &full_bar[s]);
+                } else {
+                    // token dropping: the tile's rows come from the kept runs it overlaps, one copy per run
+                    for (int r = 0; r < p.n_runs; ++r) {
+                        const int64_t a = max(j0, p.run_pos[r]), b = min(j0 + nt, p.run_pos[r + 1]);
+                        if (a < b)
+                            bulk_load(st + (size_t)(a - j0) * row_bytes,
+                                      plane + (p.run_first[r] + (a - p.run_pos[r])) * p.c,
+                                      (uint32_t)(b - a) * row_bytes, &full_bar[s]);
+                    }
+                }
             }
             ++unit;
         };

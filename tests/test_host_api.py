@@ -131,3 +131,20 @@ def test_product_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f
+
+
+def test_kept_runs_match_the_oracle(kvh):
+    import oracle
+    for N, a, b in [(1000, 4, 252), (1000, 0, 10), (1000, 10, 0), (100, 60, 40), (100, 80, 40), (5, 0, 0), (7, 7, 0),
+                    (1 << 40, 4, 1 << 20)]:
+        runs, kept = kvh.keep_sinks_and_recent(N, a, b)
+        got = [(int(r["first"]), int(r["count"])) for r in runs]
+        if a == 0 and b == 0:
+            assert got == [] and kept == 0
+            continue
+        assert got == oracle.keep_sinks_and_recent(N, a, b)
+        assert kept == sum(n for _, n in got)
+    with pytest.raises(kvh.KvhError):
+        kvh.keep_sinks_and_recent(0, 1, 1)
+    with pytest.raises(kvh.KvhError):
+        kvh.keep_sinks_and_recent(10, -1, 1)
