@@ -182,6 +182,21 @@ kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes,
                             const int32_t *page_table, int64_t page_table_len,
                             const kvh_pool *pool, int32_t *dev_status, void *stream);
 
+/* Transcode stored chunks to a coarser level on the device ("compress furthermore" in the
+ * paper's marginal-utility step, applied to an entry that is already stored).  Chunk i is read at
+ * in_streams + in_descs[i].stream_off at level in_descs[i].level and written at out_streams +
+ * out_descs[i].stream_off at level out_descs[i].level; the result is, bit for bit, the encoding at
+ * the new level of the bf16 values the old chunk decodes to.  Both descriptor arrays [device,
+ * n_chunks] must agree on n_tok, and the new level must be coarser (greater) than the old one;
+ * chunks that break a rule are skipped and reported through *dev_status (pt_off is not used).
+ * level_in / level_out: when every chunk goes from one level to one other level, pass them and a
+ * kernel specialised for the pair runs (chunks with other levels are skipped and reported);
+ * pass -1 / -1 for any mix.  The two buffers must not overlap.  n_channels <= 1024. */
+kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, const kvh_chunk_desc *in_descs,
+                         void *out_streams, uint64_t out_capacity, const kvh_chunk_desc *out_descs,
+                         int n_chunks, int n_layers, int n_channels, int level_in, int level_out,
+                         int32_t *dev_status, void *stream);
+
 /* ---- host-tier entry points: the stored form lives in (pinned) host memory ------------------
  *
  * The paper keeps compressed entries in DRAM and SSD and loads them on a hit; its loading delay

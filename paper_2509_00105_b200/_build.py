@@ -12,7 +12,7 @@ LIB = PKG / "libkvh.so"
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared",
+    "-Xcompiler", "-fPIC",
 ]
 
 
@@ -33,10 +33,22 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, f"-I{ROOT / 'include'}", f"-I{CSRC}", "-o", str(tmp), *map(str, sources())]
+    objdir = PKG / "_build"
+    objdir.mkdir(exist_ok=True)
+    common = [nvcc, *NVCC_FLAGS, f"-I{ROOT / 'include'}", f"-I{CSRC}"]
     if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    subprocess.run(cmd, check=True)
+        common.insert(1, "-Xptxas=-v")
+    # one compiler process per translation unit, side by side; then one link
+    jobs = []
+    for src in sources():
+        obj = objdir / (src.stem + f".{os.getpid()}.o")
+        jobs.append((obj, subprocess.Popen([*common, "-c", "-o", str(obj), str(src)])))
+    failed = [str(obj) for obj, proc in jobs if proc.wait() != 0]
+    if failed:
+        raise RuntimeError(f"nvcc failed for {failed}")
+    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
+    subprocess.run([nvcc, "-shared", "-o", str(tmp), *[str(obj) for obj, _ in jobs]], check=True)
+    for obj, _ in jobs:
+        obj.unlink()
     os.replace(tmp, LIB)
     return LIB

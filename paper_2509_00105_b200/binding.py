@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.kvh_keep_sinks_and_recent.argtypes = [i64, i64, i64, vp, ip, ctypes.POINTER(i64)]
         L.kvh_encode_kept.restype = i32
         L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, vp, u64, vp, vp]
+        L.kvh_transcode.restype = i32
+        L.kvh_transcode.argtypes = [vp, u64, vp, vp, u64, vp, i32, i32, i32, i32, i32, vp, vp]
         L.kvh_load_host_static.restype = i32
         L.kvh_load_host_static.argtypes = [vp, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp, u64, vp, vp]
         _lib = L
@@ -297,3 +299,17 @@ def encode_kept(kv: torch.Tensor, runs, descs_dev: torch.Tensor, n_chunks: int, 
     assert r.dtype == RUN_DTYPE
     _check(lib().kvh_encode_kept(kv.data_ptr(), l, N, c, r.ctypes.data, len(r), descs_dev.data_ptr(), n_chunks,
                                  out.data_ptr(), out.numel(), _ptr(dev_status), _stream()), "kvh_encode_kept")
+
+
+def transcode(in_streams: torch.Tensor, in_descs_dev: torch.Tensor, out_streams: torch.Tensor,
+              out_descs_dev: torch.Tensor, n_chunks: int, n_layers: int, n_channels: int,
+              level_in: int = -1, level_out: int = -1, dev_status: torch.Tensor | None = None) -> None:
+    """Re-encode stored chunks at a coarser level on the device.  level_in/level_out name the one
+    pair of levels all chunks share, or -1/-1 for a mix taken from the descriptors."""
+    assert in_streams.is_cuda and in_streams.dtype == torch.uint8
+    assert out_streams.is_cuda and out_streams.dtype == torch.uint8
+    assert in_descs_dev.numel() >= 24 * n_chunks and out_descs_dev.numel() >= 24 * n_chunks
+    _check(lib().kvh_transcode(in_streams.data_ptr(), in_streams.numel(), in_descs_dev.data_ptr(),
+                               out_streams.data_ptr(), out_streams.numel(), out_descs_dev.data_ptr(), n_chunks,
+                               n_layers, n_channels, level_in, level_out, _ptr(dev_status), _stream()),
+           "kvh_transcode")

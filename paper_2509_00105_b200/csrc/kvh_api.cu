@@ -13,6 +13,7 @@
 #include "kvh_encode.cuh"
 #include "kvh_encode_tma.cuh"
 #include "kvh_format.cuh"
+#include "kvh_host.cuh"
 
 #ifndef KVH_ENCODE_GROUPS
 #define KVH_ENCODE_GROUPS 1     // consumer groups of 256 threads in the TMA-fed encode kernel
@@ -21,39 +22,6 @@
 using namespace kvh;
 
 namespace {
-
-bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
-
-kvh_status check_shape(int level, int l, int c)
-{
-    if (level < 0 || level >= kNumLevels) return KVH_ERR_BAD_LEVEL;
-    if (l <= 0 || c <= 0 || c % kGroup != 0) return KVH_ERR_BAD_SHAPE;
-    return KVH_OK;
-}
-
-kvh_status check_pool(const kvh_pool *pool)
-{
-    if (!pool || !pool->base) return KVH_ERR_INVALID_ARG;
-    if (pool->n_layers <= 0 || pool->n_channels <= 0 || pool->n_channels % kGroup != 0) return KVH_ERR_BAD_SHAPE;
-    if (pool->page_tokens <= 0 || kChunkTokens % pool->page_tokens != 0) return KVH_ERR_BAD_SHAPE;
-    if (pool->num_pages <= 0) return KVH_ERR_BAD_SHAPE;
-    if (pool->layer_stride < 0 || pool->kv_stride < 0 || pool->page_stride < 0) return KVH_ERR_BAD_SHAPE;
-    if (!aligned(pool->base, 16) || pool->layer_stride % 8 || pool->kv_stride % 8 || pool->page_stride % 8)
-        return KVH_ERR_MISALIGNED;
-    return KVH_OK;
-}
-
-// one CTA per (chunk, layer, K|V, tile); 0 if the grid would not fit
-unsigned grid_for(int64_t n_chunks, int l)
-{
-    const int64_t g = n_chunks * l * 2 * kTilesPerChunk;
-    return (g <= 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;
-}
-
-kvh_status launch_status()
-{
-    return cudaPeekAtLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;
-}
 
 kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, void *stream)
 {

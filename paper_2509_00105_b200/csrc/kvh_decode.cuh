@@ -174,7 +174,7 @@ __device__ __forceinline__ void decode_tile(const DecodeParams &p, const uint8_t
     }
 }
 
-__global__ void __launch_bounds__(kThreads) decode_kernel(const DecodeParams p)
+static __global__ void __launch_bounds__(kThreads) decode_kernel(const DecodeParams p)
 {
     uint32_t b = blockIdx.x;
     const int tile = b % kTilesPerChunk;  b /= kTilesPerChunk;

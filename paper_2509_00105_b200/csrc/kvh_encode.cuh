@@ -279,7 +279,7 @@ __device__ __forceinline__ void encode_tile_v(const uint16_t *src, uint8_t *meta
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams p)
+static __global__ void __launch_bounds__(kThreads, 2) encode_kernel(const EncodeParams p)
 {
     __shared__ uint4 xchg[2][kThreads];                   // K: partial ranges of the two row halves
     uint32_t b = blockIdx.x;

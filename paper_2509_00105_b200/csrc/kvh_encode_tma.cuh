@@ -55,12 +55,14 @@ __device__ __forceinline__ void biased_pair(uint32_t w, f32x2 lo2, f32x2 inv2, u
     uint32_t a = w << 16, b = w & 0xffff0000u;
     if (MASKED) { a &= mask_a; b &= mask_b; }
     const f32x2 magic = f2_from_bits(0x4b000000u, 0x4b000000u);
-    // The product must be rounded before 2^23 is added.  A packed mul followed by a packed add gets
-    // contracted into one fused multiply-add by the assembler (even with .rn on both), which skips
-    // that rounding and moves about one code in a thousand; written as fma(s, 1, 2^23) the addition
-    // cannot absorb the multiply and rounds s + 2^23 once, exactly like an add.
+    // The product must be rounded before 2^23 is added.  The assembler contracts a packed mul
+    // followed by a packed add into one fused multiply-add even with .rn on both, which skips that
+    // rounding and moves a code wherever the product rounds to a tie; it does the same to
+    // fma(s, 1.0, 2^23) once it has folded the literal 1.0 away.  With a multiplier it cannot know,
+    // the fma stays: it rounds s * 1 + 2^23 once, exactly like an add, and cannot absorb the mul.
     const f32x2 s = f2_mul(f2_sub(f2_from_bits(a, b), lo2), inv2);
-    f2_bits(f2_fma(s, f2_from_bits(0x3f800000u, 0x3f800000u), magic), ta, tb);
+    const float one = kRuntimeOne;
+    f2_bits(f2_fma(s, f2_make(one, one), magic), ta, tb);
 }
 
 // Four biased codes (0x4b000000 + q) into the low 4 * BITS bits.  For 2 and 4 bits the biases end
@@ -142,22 +144,13 @@ __device__ __forceinline__ bool enc_params_k(uint32_t mn01, uint32_t mn23, uint3
     return all_quantised;
 }
 
-// A full tile: all 32 rows of the thread's 4 channels in registers, one pass over shared memory.
+// A full tile of K once its 32 rows of the thread's 4 channels (column cq) sit in registers:
+// ranges, metadata, codes.
 template <int BITS, int C>
-__device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
-                                              int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+__device__ __forceinline__ void enc_process_k(uint2 (&x)[kTileTokens], int c_rt, int cq, int tile,
+                                              uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int c = C ? C : c_rt;
-    const int C4 = c >> 2;                               // 4-channel columns per row, <= 256
-    const bool active = tid < C4;
-    const int cq = active ? tid : 0;
-    const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
-    uint2 x[kTileTokens];
-#pragma unroll
-    for (int t = 0; t < kTileTokens; ++t) x[t] = col[t * C4];
-    enc_release(empty_bar);
-    if (!active) return;
-
     uint32_t mn01 = x[0].x, mn23 = x[0].y, mx01 = x[0].x, mx23 = x[0].y;
 #pragma unroll
     for (int t = 1; t < kTileTokens; ++t) {
@@ -185,33 +178,58 @@ __device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int t
         enc_store_row_k<BITS, false>(x[t], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
 }
 
-// The last, short tile of a chunk (nt < 32 rows): rare, so two plain passes over shared memory.
+// A full tile: all 32 rows of the thread's 4 channels in registers, one pass over shared memory.
+template <int BITS, int C>
+__device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                              int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int C4 = c >> 2;                               // 4-channel columns per row, <= 256
+    const bool active = tid < C4;
+    const int cq = active ? tid : 0;
+    const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
+    uint2 x[kTileTokens];
+#pragma unroll
+    for (int t = 0; t < kTileTokens; ++t) x[t] = col[t * C4];
+    enc_release(empty_bar);
+    if (active) enc_process_k<BITS, C>(x, c_rt, cq, tile, meta_sec, codes_sec);
+}
+
+// The last, short tile of a chunk (nt < 32 rows): rare, so two plain passes over the rows.
+// row(t) returns row t of the thread's 4 channels (column cq) as two packed bf16 pairs.
+template <int BITS, typename RowFn>
+__device__ __forceinline__ void enc_k_short(RowFn row, int c, int cq, int nt, int tile,
+                                            uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const uint2 x0 = row(0);
+    uint32_t mn01 = x0.x, mn23 = x0.y, mx01 = mn01, mx23 = mn23;
+#pragma unroll 1
+    for (int t = 1; t < nt; ++t) {
+        const uint2 x = row(t);
+        mn01 = bmin2(mn01, x.x); mx01 = bmax2(mx01, x.x);
+        mn23 = bmin2(mn23, x.y); mx23 = bmax2(mx23, x.y);
+    }
+    float lo[4], inv[4];
+    uint32_t mask[4];
+    (void)enc_params_k<BITS>(mn01, mn23, mx01, mx23,
+                             reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
+    const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
+    const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
+    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
+    uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
+#pragma unroll 1
+    for (int t = 0; t < nt; ++t)
+        enc_store_row_k<BITS, true>(row(t), lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
+}
+
 template <int BITS>
 __device__ __noinline__ void enc_consume_k_short(const uint8_t *st, int c, int tid, uint64_t *empty_bar,
                                                  int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int C4 = c >> 2;
     if (tid < C4) {
-        const int cq = tid;
-        const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
-        uint32_t mn01 = col[0].x, mn23 = col[0].y, mx01 = mn01, mx23 = mn23;
-#pragma unroll 1
-        for (int t = 1; t < nt; ++t) {
-            const uint2 x = col[t * C4];
-            mn01 = bmin2(mn01, x.x); mx01 = bmax2(mx01, x.x);
-            mn23 = bmin2(mn23, x.y); mx23 = bmax2(mx23, x.y);
-        }
-        float lo[4], inv[4];
-        uint32_t mask[4];
-        (void)enc_params_k<BITS>(mn01, mn23, mx01, mx23,
-                                 reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
-        const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
-        const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
-        const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-        uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
-#pragma unroll 1
-        for (int t = 0; t < nt; ++t)
-            enc_store_row_k<BITS, true>(col[t * C4], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
+        const uint2 *col = reinterpret_cast<const uint2 *>(st) + tid;
+        enc_k_short<BITS>([&](int t) { return col[t * C4]; }, c, tid, nt, tile, meta_sec, codes_sec);
     }
     enc_release(empty_bar);
 }
@@ -235,8 +253,8 @@ __device__ __forceinline__ void enc_unrotate(uint32_t (&p)[4][W], int rot)
 }
 
 // One group: range, metadata word, codes.  x[j] is the 16-byte piece number (j + rot) & 3 of the
-// group's 64 bytes.
-template <int BITS>
+// group's 64 bytes (ROTATED), or simply piece j.
+template <int BITS, bool ROTATED = true>
 __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32_t *meta_out, uint8_t *codes_out)
 {
     uint32_t mn = bmin2(bmin2(x[0].x, x[0].y), bmin2(x[0].z, x[0].w));
@@ -269,7 +287,7 @@ __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32
             if constexpr (BITS == 4) p[j][0] = __byte_perm(a, b, 0x5410);
             if constexpr (BITS == 2) p[j][0] = __byte_perm(a, b, 0x0040);     // 16 bits; the upper half is dropped below
         }
-        enc_unrotate<W>(p, rot);
+        if (ROTATED) enc_unrotate<W>(p, rot);
     } else {                                             // a flat group: every code is 0
 #pragma unroll
         for (int j = 0; j < 4; ++j)

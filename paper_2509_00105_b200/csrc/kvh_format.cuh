@@ -149,6 +149,10 @@ __device__ __forceinline__ f32x2 f2_fma(f32x2 a, f32x2 b, f32x2 c)
     return r;
 }
 
+// 1.0f that the compiler cannot see through (constant memory may be rewritten from the host, so
+// its value is not known at compile time).  See biased_pair() for what depends on that.
+static __constant__ float kRuntimeOne = 1.0f;
+
 // Order-preserving 16-bit keys for two packed bf16: numeric order, -0 below +0.
 __device__ __forceinline__ uint32_t order_keys2(uint32_t pair)
 {

@@ -1,0 +1,400 @@
+// Transcoding kernel: a stored chunk at level m becomes a stored chunk at a coarser level n > m
+// without its bf16 values ever touching HBM.
+//
+// The policy's marginal-utility step may decide to "compress furthermore" an entry that is already
+// in storage.  What is stored is all there is to compress, so the result is defined as the
+// encoding at level n of the values the level-m chunk decodes to.  Per element the kernel reads
+// (b_m + 1)/8 bytes and writes (b_n + 1)/8 bytes; a decode into a bf16 buffer followed by an encode
+// would move 4 more.
+//
+// Structure: the encode kernel's pipeline (3 shared-memory stages fed by 1-D bulk copies, tiles
+// handed out through cluster launch control, 8 consumer warps) with the decode kernel's unpacking
+// in front.  A K thread dequantises the 32 rows of its 4 channels into packed bf16 registers and
+// continues exactly like the encoder; a V thread dequantises one whole 32-channel group.  A
+// level-0 source is the encoder itself reading the chunk's raw rows.
+#pragma once
+
+#include "kvh_async.cuh"
+#include "kvh_decode_tma.cuh"
+#include "kvh_encode_tma.cuh"
+#include "kvh_format.cuh"
+
+namespace kvh {
+
+struct TranscodeParams {
+    const uint8_t *in;
+    uint64_t in_bytes;
+    const kvh_chunk_desc *in_descs;     // device, n_chunks
+    uint8_t *out;
+    uint64_t out_capacity;
+    const kvh_chunk_desc *out_descs;    // device, n_chunks
+    int32_t l, c;
+    int32_t *status;
+};
+
+struct TcUnit {
+    EncUnit e;             // what the encoder needs (bits = the output level's)
+    int32_t bits_in;       // 16, 8, 4, 2
+};
+
+// Offset of a unit's metadata in its stage; the codes (or raw rows) start at 0.
+__host__ __device__ __forceinline__ uint32_t tc_meta_off(int c) { return 32u * (uint32_t)c; }
+
+// q_i * 2^pos(i) for the 4 codes of one K row of a 4-channel column: x[0] = elements 0, 1 and
+// x[1] = elements 2, 3 (see spread8()).
+template <int BITS>
+__device__ __forceinline__ void spread4(const uint8_t *src, f32x2 (&x)[2])
+{
+    constexpr uint32_t magic = 0x4b000000u;
+    uint32_t m[4];
+    if constexpr (BITS == 2) {
+        const uint32_t wm = (uint32_t)*src | magic;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = wm & ((3u << (2 * i)) | magic);
+    } else if constexpr (BITS == 4) {
+        const uint32_t wm = (uint32_t)*reinterpret_cast<const uint16_t *>(src) | magic;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = wm & ((15u << (4 * i)) | magic);
+    } else {
+        const uint32_t w = *reinterpret_cast<const uint32_t *>(src);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m[i] = __byte_perm(w, magic, 0x7440 + i);
+    }
+    const f32x2 bias = f2_from_bits(magic, magic);
+    x[0] = f2_sub(f2_from_bits(m[0], m[1]), bias);
+    x[1] = f2_sub(f2_from_bits(m[2], m[3]), bias);
+}
+
+// Decode parameters of a thread's 4 K channels (metadata words in shared memory), with the scale
+// pre-multiplied by 2^-position as the decode kernel does.
+template <int BIN>
+__device__ __forceinline__ void tc_params_k(const uint8_t *meta, int cq, f32x2 (&lo)[2], f32x2 (&sc)[2])
+{
+    const uint4 w4 = *reinterpret_cast<const uint4 *>(meta + 16 * (size_t)cq);
+    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    float l1[4], s1[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        decode_params<BIN>(w[i], l1[i], s1[i]);
+        s1[i] = __fmul_rn(s1[i], Pos<BIN>::prescale(i));
+    }
+    lo[0] = f2_make(l1[0], l1[1]); lo[1] = f2_make(l1[2], l1[3]);
+    sc[0] = f2_make(s1[0], s1[1]); sc[1] = f2_make(s1[2], s1[3]);
+}
+
+// One dequantised K row of a 4-channel column as two packed bf16 pairs.
+template <int BIN>
+__device__ __forceinline__ uint2 tc_row_k(const uint8_t *codes, const f32x2 (&lo)[2], const f32x2 (&sc)[2])
+{
+    f32x2 q[2];
+    spread4<BIN>(codes, q);
+    uint32_t a, b, c2, d;
+    f2_bits(f2_fma(q[0], sc[0], lo[0]), a, b);
+    f2_bits(f2_fma(q[1], sc[1], lo[1]), c2, d);
+    return make_uint2(pack_bf16x2_rn(__uint_as_float(a), __uint_as_float(b)),
+                      pack_bf16x2_rn(__uint_as_float(c2), __uint_as_float(d)));
+}
+
+template <int BIN, int BOUT, int C>
+__device__ __forceinline__ void tc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                             int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int C4 = c >> 2;
+    const bool active = tid < C4;
+    const int cq = active ? tid : 0;
+    f32x2 lo[2], sc[2];
+    tc_params_k<BIN>(st + tc_meta_off(c), cq, lo, sc);
+    const uint32_t row_bytes = (uint32_t)c * BIN / 8;
+    const uint8_t *src = st + (size_t)cq * BIN / 2;       // 4 codes = BIN / 2 bytes
+    uint2 x[kTileTokens];
+#pragma unroll
+    for (int t = 0; t < kTileTokens; ++t) x[t] = tc_row_k<BIN>(src + (size_t)t * row_bytes, lo, sc);
+    enc_release(empty_bar);
+    if (active) enc_process_k<BOUT, C>(x, c_rt, cq, tile, meta_sec, codes_sec);
+}
+
+template <int BIN, int BOUT>
+__device__ __noinline__ void tc_consume_k_short(const uint8_t *st, int c, int tid, uint64_t *empty_bar,
+                                                int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    if (tid < (c >> 2)) {
+        f32x2 lo[2], sc[2];
+        tc_params_k<BIN>(st + tc_meta_off(c), tid, lo, sc);
+        const uint32_t row_bytes = (uint32_t)c * BIN / 8;
+        const uint8_t *src = st + (size_t)tid * BIN / 2;
+        enc_k_short<BOUT>([&](int t) { return tc_row_k<BIN>(src + (size_t)t * row_bytes, lo, sc); },
+                          c, tid, nt, tile, meta_sec, codes_sec);
+    }
+    enc_release(empty_bar);
+}
+
+// V: a thread dequantises whole groups (32 codes, one metadata word) and encodes them again.
+template <int BIN, int BOUT, int C>
+__device__ __forceinline__ void tc_consume_v(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+                                             int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int c = C ? C : c_rt;
+    const int gpr = c >> 5;
+    const int ngroups = nt * gpr;
+    const uint32_t *meta_in = reinterpret_cast<const uint32_t *>(st + tc_meta_off(c));
+    const size_t g_first = (size_t)tile * kTileTokens * gpr;
+    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec) + g_first;
+    uint8_t *codes = codes_sec + g_first * (4 * BOUT);
+    constexpr int U = 2;
+    const int iters = (ngroups + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);  // the same for every thread
+    for (int it = 0; it < iters; ++it) {
+        const int g0 = it * kEncGroupThreads * U + tid;
+        uint4 x[U][4];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int g = g0 + k * kEncGroupThreads;
+            if (g < ngroups) {
+                float l1, s0;
+                decode_params<BIN>(meta_in[g], l1, s0);
+                const f32x2 sa = f2_make(__fmul_rn(s0, Pos<BIN>::prescale(0)), __fmul_rn(s0, Pos<BIN>::prescale(1)));
+                const f32x2 sb = f2_make(__fmul_rn(s0, Pos<BIN>::prescale(2)), __fmul_rn(s0, Pos<BIN>::prescale(3)));
+                const f32x2 ll = f2_make(l1, l1);
+                const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+                const uint8_t *src = st + (size_t)g * (4 * BIN);       // 32 codes = 4 * BIN bytes
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    f32x2 q[4];
+                    spread8<BIN>(src + j * BIN, q);
+                    x[k][j] = fma_pack8(q, sc, lo);
+                }
+            }
+        }
+        if (it == iters - 1) enc_release(empty_bar);
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int g = g0 + k * kEncGroupThreads;
+            if (g < ngroups) enc_group_v<BOUT, false>(x[k], 0, meta + g, codes + (size_t)g * (4 * BOUT));
+        }
+    }
+}
+
+// One unit with both levels known at compile time (LOUT > LIN).
+template <int C, int LIN, int LOUT>
+__device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_t *st, int c_rt, int tid,
+                                                  uint64_t *eb)
+{
+    if constexpr (LIN == 0) {
+        enc_consume_level<C, LOUT>(u, st, c_rt, tid, eb);            // raw rows: the encoder as it is
+    } else {
+        constexpr int BIN = 16 >> LIN, BOUT = 16 >> LOUT;
+        if (u.kv) tc_consume_v<BIN, BOUT, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        else if (u.nt == kTileTokens) tc_consume_k<BIN, BOUT, C>(st, c_rt, tid, eb, u.tile, u.meta, u.codes);
+        else tc_consume_k_short<BIN, BOUT>(st, C ? C : c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+    }
+}
+template <int C, int LIN, int LOUT>
+__device__ __noinline__ void tc_consume_levels_call(const EncUnit *u, const uint8_t *st, int c_rt, int tid,
+                                                    uint64_t *eb)
+{
+    tc_consume_levels<C, LIN, LOUT>(*u, st, c_rt, tid, eb);
+}
+
+// LIN, LOUT >= 0: every chunk goes from LIN to LOUT (checked by the producer); -1: any mix.
+template <int C, int LIN, int LOUT>
+__device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, int c_rt, int tid, uint64_t *eb)
+{
+    if constexpr (LIN >= 0) {
+        tc_consume_levels<C, LIN, LOUT>(u.e, st, c_rt, tid, eb);
+    } else {
+        switch (u.bits_in * 16 + u.e.bits) {             // uniform per consumer group
+        case 16 * 16 + 8: tc_consume_levels_call<C, 0, 1>(&u.e, st, c_rt, tid, eb); break;
+        case 16 * 16 + 4: tc_consume_levels_call<C, 0, 2>(&u.e, st, c_rt, tid, eb); break;
+        case 16 * 16 + 2: tc_consume_levels_call<C, 0, 3>(&u.e, st, c_rt, tid, eb); break;
+        case 8 * 16 + 4: tc_consume_levels_call<C, 1, 2>(&u.e, st, c_rt, tid, eb); break;
+        case 8 * 16 + 2: tc_consume_levels_call<C, 1, 3>(&u.e, st, c_rt, tid, eb); break;
+        default: tc_consume_levels_call<C, 2, 3>(&u.e, st, c_rt, tid, eb); break;
+        }
+    }
+}
+
+// sched as in the encode kernel.  One CTA per SM: 8 consumer warps and a producer warp.
+template <int C, int LIN, int LOUT>
+__global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
+transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sched)
+{
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    __shared__ __align__(8) uint64_t full_bar[kEncStages];
+    __shared__ __align__(8) uint64_t empty_bar[kEncStages];
+    __shared__ TcUnit info[kEncStages];
+    __shared__ int abort_flag;
+    __shared__ __align__(16) uint4 clc_response[2];
+    __shared__ __align__(8) uint64_t clc_bar[2];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kProducerWarp = kEncGroupThreads / 32;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kEncStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kEncGroupThreads / 32);
+        }
+        mbar_init(&clc_bar[0], 1);
+        mbar_init(&clc_bar[1], 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kProducerWarp) {
+        // ------------------------------ producer warp ------------------------------
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        uint32_t unit = 0;
+        bool ok = true;
+        int cur_chunk = -1;
+        bool valid = false;
+        kvh_chunk_desc di{}, dout{};
+        LayerLayout Li = layer_layout(0, p.c, 1), Lo = Li;
+
+        auto acquire = [&]() -> bool {                   // wait until the unit's stage is free
+            const int s = unit % kEncStages;
+            if (unit < (uint32_t)kEncStages) return true;
+            bool w = true;
+            if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / kEncStages) - 1) & 1, &abort_flag);
+            return __shfl_sync(0xffffffffu, w, 0);
+        };
+
+        auto do_tile = [&](int64_t tile_id) {
+            const int tile = (int)(tile_id % kTilesPerChunk);
+            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int kv = (int)(plane_id & 1);
+            const int layer = (int)((plane_id >> 1) % p.l);
+            const int chunk = (int)((plane_id >> 1) / p.l);
+            if (chunk != cur_chunk) {
+                cur_chunk = chunk;
+                di = p.in_descs[chunk];
+                dout = p.out_descs[chunk];
+                int err = check_desc(di, p.l, p.c, p.in_bytes);
+                if (err == KVH_OK) err = check_desc(dout, p.l, p.c, p.out_capacity);
+                if (err == KVH_OK && di.n_tok != dout.n_tok) err = KVH_ERR_BAD_SHAPE;
+                if (err == KVH_OK && dout.level <= di.level) err = KVH_ERR_BAD_LEVEL;   // only towards coarser levels
+                if (err == KVH_OK && LIN >= 0 && (di.level != LIN || dout.level != LOUT)) err = KVH_ERR_BAD_LEVEL;
+                valid = err == KVH_OK;
+                if (!valid) {
+                    if (lane == 0) report(p.status, err);
+                } else {
+                    Li = layer_layout(di.level, p.c, di.n_tok);
+                    Lo = layer_layout(dout.level, p.c, dout.n_tok);
+                }
+            }
+            if (!valid) return;
+            const int n = di.n_tok;
+            const int t0 = tile * kTileTokens;
+            const int nt = min(kTileTokens, n - t0);
+            if (nt <= 0) return;
+            const uint8_t *lay_in = p.in + di.stream_off + (uint64_t)layer * Li.layer_bytes();
+            uint8_t *lay_out = p.out + dout.stream_off + (uint64_t)layer * Lo.layer_bytes();
+            ok = acquire();
+            if (!ok) return;
+            if (lane == 0) {
+                const int s = unit % kEncStages;
+                TcUnit &u = info[s];
+                u.bits_in = level_bits(di.level);
+                u.e.bits = level_bits(dout.level); u.e.kv = kv; u.e.nt = nt; u.e.tile = tile;
+                u.e.last = t0 + nt == n;
+                u.e.meta_payload = (uint32_t)(kv ? Lo.vmeta_payload : Lo.kmeta_payload);
+                u.e.meta_padded = (uint32_t)(kv ? Lo.vmeta : Lo.kmeta);
+                u.e.codes_payload = (uint32_t)Lo.codes_payload;
+                u.e.codes_padded = (uint32_t)Lo.kcodes;
+                u.e.meta = lay_out + Lo.meta_off(kv);
+                u.e.codes = lay_out + Lo.codes_off(kv);
+                uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+                const uint8_t *codes_in = lay_in + Li.codes_off(kv);
+                if (di.level == 0) {
+                    const uint32_t bytes = 2u * (uint32_t)nt * (uint32_t)p.c;
+                    mbar_arrive_expect_tx(&full_bar[s], bytes);
+                    bulk_load(st, codes_in + 2 * (uint64_t)t0 * p.c, bytes, &full_bar[s]);
+                } else {
+                    const int b = level_bits(di.level);
+                    const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
+                    const uint8_t *meta_in = lay_in + Li.meta_off(kv);
+                    const uint8_t *msrc = kv == 0 ? meta_in + 4 * (uint64_t)tile * p.c
+                                                  : meta_in + 4 * (uint64_t)t0 * (p.c / kGroup);
+                    const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * (p.c / kGroup));
+                    mbar_arrive_expect_tx(&full_bar[s], cbytes + mbytes);
+                    bulk_load(st, codes_in + (uint64_t)t0 * p.c * b / 8, cbytes, &full_bar[s]);
+                    bulk_load(st + tc_meta_off(p.c), msrc, mbytes, &full_bar[s]);
+                }
+            }
+            ++unit;
+        };
+
+        int64_t tile_id = blockIdx.x;
+        uint32_t query = 0;                              // answers asked for so far
+        bool asked = false;                              // one answer still outstanding
+        while (ok && tile_id < total_tiles) {
+            if (sched == 1) {                            // ask for the next tile while this one streams
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&clc_bar[query & 1], 16);
+                    clc_try_cancel(&clc_response[query & 1], &clc_bar[query & 1]);
+                }
+                asked = true;
+            }
+            do_tile(tile_id);
+            if (!ok) break;
+            if (sched == 1) {
+                uint32_t got = 0, next = 0, w = 1;
+                if (lane == 0) {
+                    w = mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &abort_flag);
+                    if (w) got = clc_query(&clc_response[query & 1], next);
+                }
+                w = __shfl_sync(0xffffffffu, w, 0);
+                got = __shfl_sync(0xffffffffu, got, 0);
+                next = __shfl_sync(0xffffffffu, next, 0);
+                if (!w) { ok = false; break; }
+                asked = false;
+                ++query;
+                if (!got) break;                         // no CTA left to take over: never ask again
+                tile_id = next;
+            } else {
+                tile_id += gridDim.x;
+            }
+        }
+        if (ok) ok = acquire();
+        if (ok) {                                        // end marker
+            if (lane == 0) {
+                info[unit % kEncStages].e.bits = 0;
+                mbar_arrive(&full_bar[unit % kEncStages]);
+            }
+            ++unit;
+        }
+        if (!ok && lane == 0) {
+            report(p.status, KVH_ERR_TIMEOUT);
+            abort_flag = 1;
+        }
+        // Leave only after every copy issued has landed (see the encode kernel).
+        if (lane == 0) {
+            int never = 0;
+            const uint32_t first = unit > (uint32_t)kEncStages ? unit - kEncStages : 0;
+            for (uint32_t w = first; w < unit; ++w)
+                (void)mbar_wait(&full_bar[w % kEncStages], (w / kEncStages) & 1, &never);
+            if (asked) (void)mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &never);
+        }
+    } else {
+        // ------------------------------ consumer warps ------------------------------
+        const int tid = threadIdx.x;
+        for (uint32_t unit = 0;; ++unit) {
+            const int s = unit % kEncStages;
+            if (!mbar_wait(&full_bar[s], (unit / kEncStages) & 1, &abort_flag)) {
+                report(p.status, KVH_ERR_TIMEOUT);
+                abort_flag = 1;
+                break;
+            }
+            const TcUnit u = info[s];
+            if (u.e.bits == 0) break;
+            const uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+            if (u.e.last && tid < KVH_SECTION_ALIGN) {   // the plane's last tile clears the padding
+                if (u.e.codes_payload + tid < u.e.codes_padded) u.e.codes[u.e.codes_payload + tid] = 0;
+                if (u.e.meta_payload + tid < u.e.meta_padded) u.e.meta[u.e.meta_payload + tid] = 0;
+            }
+            tc_dispatch<C, LIN, LOUT>(u, st, p.c, tid, &empty_bar[s]);
+        }
+    }
+}
+
+}  // namespace kvh
