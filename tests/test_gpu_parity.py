@@ -284,3 +284,31 @@ def test_gpu_decodes_oracle_streams_and_oracle_decodes_gpu_streams(kvh):
         got, _ = kvh.encode(kv, level)
         wp, _ = oracle_pool(flat.numel(), strides, got.cpu().numpy(), offsets, [N], [level], l, c, ids.numpy(), 16)
         assert np.array_equal(to_np16(flat), wp)
+
+
+def lattice_kv(l, N, c, seed):
+    """Values on small integer lattices times a power of two: within a group x - min and max - min
+    are small integers, so (x - min) * qmax / (max - min) lands exactly on k + 1/2 very often while
+    qmax / (max - min) is inexact.  Any evaluation that does not round the product before rounding to
+    an integer (a fused multiply-add) then picks the wrong neighbour."""
+    rng = np.random.default_rng(seed)
+    span = rng.integers(1, 256, size=(l, 2, (N + 31) // 32, 1, c // 32, 1))          # per 32 x 32 block
+    m = rng.integers(0, 256, size=(l, 2, (N + 31) // 32, 32, c // 32, 32)) % (span + 1)
+    m[:, :, :, 0, :, 0] = 0                                   # every K column and V row of a block sees 0 ...
+    m[:, :, :, :, :, 1] = np.where(np.arange(32)[None, None, None, :, None] % 2 == 0, 0, span[..., 0])
+    m[:, :, :, 1, :, :] = np.where(np.arange(32) % 2 == 0, span[:, :, :, 0, :, :], 0)   # ... and the block's span
+    e = rng.integers(-6, 7, size=(l, 2, (N + 31) // 32, 1, c // 32, 1))
+    x = (m * (2.0 ** e)).astype(np.float32).reshape(l, 2, -1, c // 32, 32)
+    x = x.reshape(l, 2, -1, c)[:, :, :N]
+    bits = np.ascontiguousarray(x).view(np.uint32)
+    assert np.all((bits & 0xFFFF) == 0)                       # exact in bf16
+    return (bits >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("l,c,N", [(2, 1024, 512), (1, 64, 300), (1, 2048, 64)])
+@pytest.mark.parametrize("level", [1, 2, 3])
+def test_encode_rounds_ties_like_the_oracle(kvh, l, c, N, level):
+    kv_np = lattice_kv(l, N, c, seed=level * 100 + c)
+    want, _ = oracle.encode_context(kv_np, level)
+    got, _ = kvh.encode(from_np16(kv_np), level)
+    assert np.array_equal(got.cpu().numpy(), want)

@@ -114,3 +114,20 @@ def test_transcode_at_benchmark_shape(kvh):
                      pool, status)
     again, _ = kvh.encode(pool.tensor.view(l, 2, N, c), 3)
     assert torch.equal(again, out)
+
+
+@pytest.mark.parametrize("pair", PAIRS)
+def test_transcode_rounds_ties_like_the_oracle(kvh, pair):
+    """Sources on integer lattices (see lattice_kv): re-quantising hits exact ties all the time."""
+    from test_gpu_parity import lattice_kv
+    l, c, N = 2, 1024, 512
+    kv_np = lattice_kv(l, N, c, seed=17 + pair[0] * 4 + pair[1])
+    src, offsets = oracle.encode_context(kv_np, pair[0])
+    want = oracle_transcode_context(src, offsets, [256, 256], [pair[0]] * 2, [pair[1]] * 2, l, c)
+    din, _ = kvh.plan_chunks(l, c, N, pair[0])
+    dout, total = kvh.plan_chunks(l, c, N, pair[1])
+    for hint in (pair, (-1, -1)):
+        out = torch.empty(total, dtype=torch.uint8, device="cuda")
+        kvh.transcode(torch.from_numpy(src).cuda(), kvh.descs_to_tensor(din, "cuda"), out,
+                      kvh.descs_to_tensor(dout, "cuda"), 2, l, c, *hint)
+        assert np.array_equal(out.cpu().numpy(), want)
