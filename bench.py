@@ -200,6 +200,44 @@ def whole_job_gbps(world: int, bytes_per_rank: float, ms: float) -> float:
     return world * bytes_per_rank / ms / 1e6
 
 
+def time_extras(kvh, kv, plans, stream_buf, status, l, c, N, n_chunks, dev, reps: int = 5):
+    """Transcoding (every pair of levels) and token dropping (4 sink tokens + a recent window, a
+    quarter of the context kept), each as the mean of `reps` launches over the whole context after
+    one warm-up launch.  Bytes counted: streams read + streams written (transcode), kept bf16 rows
+    read + streams written (token dropping)."""
+    def timed(fn):
+        fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) / reps
+
+    elements = l * 2 * N * c
+    out = {"transcode": [], "token_dropping": []}
+    second = torch.empty(plans[1][2], dtype=torch.uint8, device=dev)
+    for lin in (0, 1, 2):
+        _, descs_in_dev, total_in = plans[lin]
+        kvh.encode(kv, lin, out=stream_buf[:total_in], dev_status=status)
+        for lout in range(lin + 1, 4):
+            _, descs_out_dev, total_out = plans[lout]
+            ms = timed(lambda: kvh.transcode(stream_buf[:total_in], descs_in_dev, second[:total_out], descs_out_dev,
+                                             n_chunks, l, c, lin, lout, dev_status=status))
+            out["transcode"].append({"from": lin, "to": lout, "ms": round(ms, 4),
+                                     "hbm_gbps": round((total_in + total_out) / ms / 1e6, 1),
+                                     "tokens_per_s": round(N / ms * 1e3)})
+    runs, n_kept = kvh.keep_sinks_and_recent(N, 4, N // 4 - 4)
+    for level in LEVELS:
+        descs, total = kvh.plan_chunks(l, c, n_kept, level)
+        ms = timed(lambda: kvh.encode_kept(kv, runs, None, len(descs), second[:total], status, level=level))
+        out["token_dropping"].append({"level": level, "kept_tokens": n_kept, "ms": round(ms, 4),
+                                      "hbm_gbps": round((2 * elements * n_kept // N + total) / ms / 1e6, 1)})
+    assert status.item() == 0
+    return out
+
+
 def run_ours(args, shape: workloads.Shape):
     import torch.distributed as dist
     import paper_2509_00105_b200 as kvh
@@ -268,6 +306,11 @@ def run_ours(args, shape: workloads.Shape):
     total_ms = times[0]
     enc_ms = dict(zip(LEVELS, times[1:5]))
     dec_ms = dict(zip(LEVELS, times[5:9]))
+
+    # ---- the two further store-side operations, timed on their own after the steps ----
+    extras = None
+    if world == 1 and not args.no_extras:
+        extras = time_extras(kvh, kv, plans, stream_buf, status, l, c, N, n_chunks, dev)
 
     # ---- end to end: stored form in pinned host memory ----
     e2e = None
@@ -352,6 +395,11 @@ def run_ours(args, shape: workloads.Shape):
     }
     if e2e is not None:
         out["e2e"] = e2e
+    if extras is not None:
+        for rows in extras.values():
+            for r in rows:
+                r["roofline_frac"] = round(r["hbm_gbps"] / peak, 4)
+        out["extras"] = extras
     if world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
         kv_np, layers = oracle_inputs(shape, cores, target_s=4.0)
@@ -375,6 +423,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the transcode / token-dropping timings")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     shape = workloads.LLAMA70B_32K

@@ -155,11 +155,15 @@ kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n
 /* Encode the kept tokens of a context.  kv [device] as for kvh_encode ([n_layers][2][n_tokens]
  * [n_channels]).  runs [host, n_runs <= KVH_MAX_KEPT_RUNS]: ascending, disjoint, inside the
  * context.  descs [device, n_chunks = ceil(n_kept / 256)] describe the chunks of the compacted
- * sequence (lay them out with kvh_plan_chunks for n_kept tokens); everything else as for
- * kvh_encode_chunks.  n_channels must not exceed 1024 (KVH_ERR_BAD_SHAPE otherwise). */
+ * sequence (lay them out with kvh_plan_chunks for n_kept tokens).  level >= 0 says that every
+ * chunk is stored at this one level: descs may then be NULL (chunk i lands at i *
+ * kvh_level_bytes(level, ..., 256), as with kvh_encode), a kernel holding only that level's code
+ * runs, and a descriptor of another level is skipped and reported; level = -1 takes a level per
+ * chunk from descs.  Everything else as for kvh_encode_chunks.  n_channels must not exceed 1024
+ * (KVH_ERR_BAD_SHAPE otherwise). */
 kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
                            const kvh_token_run *runs, int n_runs,
-                           const kvh_chunk_desc *descs, int n_chunks,
+                           const kvh_chunk_desc *descs, int n_chunks, int level,
                            void *out, uint64_t out_capacity,
                            int32_t *dev_status, void *stream);
 

@@ -81,7 +81,7 @@ def lib() -> ctypes.CDLL:
         L.kvh_keep_sinks_and_recent.restype = i32
         L.kvh_keep_sinks_and_recent.argtypes = [i64, i64, i64, vp, ip, ctypes.POINTER(i64)]
         L.kvh_encode_kept.restype = i32
-        L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, vp, u64, vp, vp]
+        L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, i32, vp, u64, vp, vp]
         L.kvh_transcode.restype = i32
         L.kvh_transcode.argtypes = [vp, u64, vp, vp, u64, vp, i32, i32, i32, i32, i32, vp, vp]
         L.kvh_load_host_static.restype = i32
@@ -290,14 +290,15 @@ def keep_sinks_and_recent(n_tokens: int, n_sink: int, n_recent: int) -> tuple[np
     return runs[:n.value].copy(), kept.value
 
 
-def encode_kept(kv: torch.Tensor, runs, descs_dev: torch.Tensor, n_chunks: int, out: torch.Tensor,
-                dev_status: torch.Tensor | None = None) -> None:
-    """Token dropping: encode only the kept runs of a context, compacted; descs_dev lays out the
-    chunks of the kept sequence (plan_chunks for n_kept tokens)."""
+def encode_kept(kv: torch.Tensor, runs, descs_dev: torch.Tensor | None, n_chunks: int, out: torch.Tensor,
+                dev_status: torch.Tensor | None = None, level: int = -1) -> None:
+    """Token dropping: encode only the kept runs of a context, compacted.  descs_dev lays out the
+    chunks of the kept sequence (plan_chunks for n_kept tokens); with one level for all chunks pass
+    `level` (descs_dev may then be None: chunks back to back) and the specialised kernel runs."""
     l, N, c = _check_kv(kv)
     r = np.ascontiguousarray(np.asarray(runs, dtype=RUN_DTYPE) if not isinstance(runs, np.ndarray) else runs)
     assert r.dtype == RUN_DTYPE
-    _check(lib().kvh_encode_kept(kv.data_ptr(), l, N, c, r.ctypes.data, len(r), descs_dev.data_ptr(), n_chunks,
+    _check(lib().kvh_encode_kept(kv.data_ptr(), l, N, c, r.ctypes.data, len(r), _ptr(descs_dev), n_chunks, level,
                                  out.data_ptr(), out.numel(), _ptr(dev_status), _stream()), "kvh_encode_kept")
 
 

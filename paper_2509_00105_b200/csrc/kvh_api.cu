@@ -86,7 +86,7 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream)
         constexpr int G = KVH_ENCODE_GROUPS;
         const size_t dyn = (size_t)kEncStages * kEncStageBytes;
         // one level for the whole launch (kvh_encode): an instance that holds only that level's code
-        const int level = p.descs ? -1 : p.level;
+        const int level = p.descs ? p.hint_level : p.level;
         void (*kernel)(const EncodeParams, const int, const int);
         if (p.c == 1024) {
             kernel = level == 0 ? encode_tma_kernel<1024, G, 0> : level == 1 ? encode_tma_kernel<1024, G, 1>
@@ -218,6 +218,7 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
     p.kv = static_cast<const uint16_t *>(kv);
     p.l = n_layers; p.c = n_channels; p.N = n_tokens; p.src_N = n_tokens;
     p.descs = descs;
+    p.hint_level = -1;
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
     p.status = dev_status;
@@ -245,11 +246,11 @@ kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n
 
 kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
                            const kvh_token_run *runs, int n_runs, const kvh_chunk_desc *descs, int n_chunks,
-                           void *out, uint64_t out_capacity, int32_t *dev_status, void *stream)
+                           int level, void *out, uint64_t out_capacity, int32_t *dev_status, void *stream)
 {
-    if (!kv || !out || !descs || !runs || n_tokens <= 0 || n_runs <= 0 || n_runs > kMaxKeptRuns)
+    if (!kv || !out || !runs || n_tokens <= 0 || n_runs <= 0 || n_runs > kMaxKeptRuns || (!descs && level < 0))
         return KVH_ERR_INVALID_ARG;
-    const kvh_status s = check_shape(0, n_layers, n_channels);
+    const kvh_status s = check_shape(level < 0 ? 0 : level, n_layers, n_channels);
     if (s != KVH_OK) return s;
     if (n_channels > kEncMaxChannels) return KVH_ERR_BAD_SHAPE;       // the gather is the TMA kernel's
     if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
@@ -269,6 +270,15 @@ kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n
     p.kv = static_cast<const uint16_t *>(kv);
     p.l = n_layers; p.c = n_channels; p.N = kept; p.src_N = n_tokens;
     p.descs = descs;
+    p.hint_level = level < 0 ? -1 : level;
+    if (!descs) {                                        // chunks back to back at the one level
+        p.level = level;
+        p.full_chunk_bytes = chunk_bytes(level, n_layers, n_channels, kChunkTokens);
+        uint64_t need = 0;
+        const kvh_status ps = kvh_plan_chunks(n_layers, n_channels, kept, nullptr, level, 0, 0, 16, nullptr, &need);
+        if (ps != KVH_OK) return ps;
+        if (need > out_capacity) return KVH_ERR_BUFFER_TOO_SMALL;
+    }
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
     p.status = dev_status;
@@ -429,6 +439,7 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
         p.kv = static_cast<const uint16_t *>(kv);
         p.l = n_layers; p.c = n_channels; p.N = n_tokens; p.src_N = n_tokens;
         p.descs = descs_dev;
+        p.hint_level = -1;
         p.chunk0 = s.first;
         p.out = static_cast<uint8_t *>(dev_staging);
         p.capacity = staging_bytes;

@@ -41,6 +41,13 @@ def test_encode_kept_matches_oracle(kvh, l, c, N, runs, levels):
     assert status.item() == 0
     assert np.array_equal(g[:total], want)
     assert np.all(g[total:] == 0xAB)
+    if isinstance(levels, int):                          # one level: the specialised kernel, with and without descriptors
+        for dd in (kvh.descs_to_tensor(descs, "cuda"), None):
+            out.fill_(0xAB)
+            kvh.encode_kept(kv, np.array(runs, dtype=kvh.RUN_DTYPE), dd, len(descs), out[:total], status, level=levels)
+            g = out.cpu().numpy()
+            assert status.item() == 0
+            assert np.array_equal(g[:total], want) and np.all(g[total:] == 0xAB)
 
     # a hit loads the kept tokens into consecutive page slots
     npg = workloads.n_pages(n_kept)
@@ -65,7 +72,7 @@ def test_sinks_and_recent_window_at_benchmark_shape(kvh):
     assert total * 4 == kvh.plan_chunks(l, c, N, 3)[1]                   # size = rate x size
     out = torch.empty(total, dtype=torch.uint8, device="cuda")
     status = new_status()
-    kvh.encode_kept(kv, runs, kvh.descs_to_tensor(descs, "cuda"), len(descs), out, status)
+    kvh.encode_kept(kv, runs, None, len(descs), out, status, level=3)
     assert status.item() == 0
     compact = torch.cat([kv[:, :, :4], kv[:, :, N - 2044:]], dim=2)
     for i in (0, 3, 7):                                  # chunk 0 holds the seam
@@ -91,6 +98,16 @@ def test_encode_kept_rejects_bad_runs(kvh):
     out.fill_(0xEE)
     kvh.encode_kept(kv, R([(0, 99)]), dd, len(descs), out, status)
     assert status.item() == 3 and bool((out == 0xEE).all())
+    # a level is announced and a descriptor has another one
+    status = new_status()
+    kvh.encode_kept(kv, R([(0, 100)]), dd, len(descs), out, status, level=2)
+    assert status.item() == 2
+    with pytest.raises(kvh.KvhError) as e:               # neither descriptors nor a level
+        kvh.encode_kept(kv, R([(0, 100)]), None, len(descs), out)
+    assert e.value.status == 1
+    with pytest.raises(kvh.KvhError) as e:
+        kvh.encode_kept(kv, R([(0, 100)]), None, len(descs), out[:total - 128], level=1)
+    assert e.value.status == 5
     wide = workloads.make_kv(1, 40, 2048, seed=2, device="cuda")
     d2, t2 = kvh.plan_chunks(1, 2048, 8, 1)
     with pytest.raises(kvh.KvhError) as e:
