@@ -230,6 +230,40 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
                           int32_t *dev_status, int32_t *host_status, uint64_t slice_bytes,
                           void *copy_stream, void *stream);
 
+/* ---- the policy: which stored form every entry gets ---------------------------------------------
+ *
+ * Host arithmetic only.  The paper's Design section: Utility(i) = Freq(i) * (alpha * Quality(i, M_i,
+ * R_i) - size(i, M_i, R_i) / Bandwidth); the choice of (M_i, R_i) under a tier's capacity is a
+ * multiple-choice knapsack, solved greedily by the smallest marginal utility drop (utility lost
+ * per byte saved) over each entry's LP-undominated options, eviction included.  An option is one
+ * stored form of an entry: its size in bytes (kvh_level_bytes / kvh_plan_chunks for the level and
+ * the kept tokens) and the estimated quality of answers generated from it.  The options of all
+ * entries are concatenated; option_begin [n_entries + 1] delimits each entry's. */
+typedef struct {
+    uint64_t size;         /* stored bytes */
+    double quality;        /* estimated quality, any scale (alpha converts it to seconds) */
+} kvh_option;
+
+typedef struct {
+    double alpha;          /* weight of quality against loading delay */
+    double bandwidth;      /* bytes per second from this tier to the GPU, > 0 */
+    uint64_t capacity;     /* bytes */
+} kvh_tier;
+
+/* One tier.  choice_out [n_entries]: index of the chosen option within the entry's own options,
+ * or -1 = evicted.  used_bytes, total_utility [host] may be NULL.  Slopes are compared in extended
+ * precision; ties go to the lower entry index. */
+kvh_status kvh_policy_assign(const double *freq, const kvh_option *options, const int32_t *option_begin,
+                             int n_entries, const kvh_tier *tier, int32_t *choice_out,
+                             uint64_t *used_bytes, double *total_utility);
+
+/* Several tiers, fastest first (DRAM, then SSD in the paper): what a tier evicts is offered to
+ * the next; what the last one evicts is recomputed on a hit.  tier_out [n_entries]: tier index or
+ * -1; choice_out as above. */
+kvh_status kvh_policy_assign_tiers(const double *freq, const kvh_option *options, const int32_t *option_begin,
+                                   int n_entries, const kvh_tier *tiers, int n_tiers,
+                                   int32_t *tier_out, int32_t *choice_out);
+
 /* ---- a load entry point that allocates nothing -------------------------------------------------
  *
  * The paper has no counterpart to this call; it exists for how the library gets deployed.  Some

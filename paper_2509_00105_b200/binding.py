@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
         L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, i32, vp, u64, vp, vp]
         L.kvh_transcode.restype = i32
         L.kvh_transcode.argtypes = [vp, u64, vp, vp, u64, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.kvh_policy_assign.restype = i32
+        L.kvh_policy_assign.argtypes = [vp, vp, vp, i32, vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_double)]
+        L.kvh_policy_assign_tiers.restype = i32
+        L.kvh_policy_assign_tiers.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp]
         L.kvh_load_host_static.restype = i32
         L.kvh_load_host_static.argtypes = [vp, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp, u64, vp, vp]
         _lib = L
@@ -314,3 +318,38 @@ def transcode(in_streams: torch.Tensor, in_descs_dev: torch.Tensor, out_streams:
                                out_streams.data_ptr(), out_streams.numel(), out_descs_dev.data_ptr(), n_chunks,
                                n_layers, n_channels, level_in, level_out, _ptr(dev_status), _stream()),
            "kvh_transcode")
+
+
+OPTION_DTYPE = np.dtype([("size", "<u8"), ("quality", "<f8")])
+TIER_DTYPE = np.dtype([("alpha", "<f8"), ("bandwidth", "<f8"), ("capacity", "<u8")])
+
+
+def _policy_args(freq, options, option_begin):
+    f = np.ascontiguousarray(freq, dtype=np.float64)
+    o = np.ascontiguousarray(options, dtype=OPTION_DTYPE)
+    b = np.ascontiguousarray(option_begin, dtype=np.int32)
+    assert b.size == f.size + 1 and b[0] == 0 and b[-1] == o.size
+    return f, o, b
+
+
+def policy_assign(freq, options, option_begin, alpha: float, bandwidth: float, capacity: int):
+    """Greedy marginal-utility choice of a stored form per entry for one tier.
+    Returns (choice per entry, -1 = evicted; bytes used; total utility)."""
+    f, o, b = _policy_args(freq, options, option_begin)
+    tier = np.array([(alpha, bandwidth, capacity)], dtype=TIER_DTYPE)
+    choice = np.empty(f.size, dtype=np.int32)
+    used, total = ctypes.c_uint64(), ctypes.c_double()
+    _check(lib().kvh_policy_assign(f.ctypes.data, o.ctypes.data, b.ctypes.data, f.size, tier.ctypes.data,
+                                   choice.ctypes.data, ctypes.byref(used), ctypes.byref(total)), "kvh_policy_assign")
+    return choice, used.value, total.value
+
+
+def policy_assign_tiers(freq, options, option_begin, tiers):
+    """The same over several tiers, fastest first; tiers: (alpha, bandwidth, capacity) each.
+    Returns (tier per entry or -1, choice per entry or -1)."""
+    f, o, b = _policy_args(freq, options, option_begin)
+    t = np.array([tuple(x) for x in tiers], dtype=TIER_DTYPE)
+    tier_out, choice = np.empty(f.size, dtype=np.int32), np.empty(f.size, dtype=np.int32)
+    _check(lib().kvh_policy_assign_tiers(f.ctypes.data, o.ctypes.data, b.ctypes.data, f.size, t.ctypes.data, len(t),
+                                         tier_out.ctypes.data, choice.ctypes.data), "kvh_policy_assign_tiers")
+    return tier_out, choice

@@ -92,3 +92,29 @@ def n_chunks(n_tokens: int) -> int:
 def n_pages(n_tokens: int) -> int:
     """Pages a context occupies; chunk i of a context starts at page slot 16*i."""
     return (n_tokens + PAGE_TOKENS - 1) // PAGE_TOKENS
+
+
+def policy_entries(n_entries: int, seed: int):
+    """Synthetic inputs of the policy: per entry a reuse frequency (Zipf-like), a length in tokens
+    (log-uniform in [2K, 32K]) and, for every stored form on offer, an estimated quality.  Stored
+    forms: quantisation level 0..3 crossed with the kept fraction of tokens (1, 1/2, 1/4, 1/8).
+    Quality falls with coarser levels and with dropped tokens, each entry with its own sensitivity
+    (some texts tolerate dropping, others quantisation); the numbers stand in for the profiled
+    quality curves the paper's estimator measures with a language model, which is not available
+    here.  Returns (freq [n], n_tokens [n], forms [(level, keep_fraction)], quality [n][len(forms)])."""
+    g = torch.Generator().manual_seed(seed)
+    rank = torch.randperm(n_entries, generator=g).to(torch.float64) + 1.0
+    freq = (10.0 / rank).tolist()
+    tokens = context_lengths(n_entries, BATCH_MIN_TOKENS, BATCH_MAX_TOKENS, seed + 1)
+    forms = [(level, keep) for keep in (1.0, 0.5, 0.25, 0.125) for level in range(4)]
+    sens_q = 0.02 + 0.25 * torch.rand(n_entries, generator=g, dtype=torch.float64)     # loss at 2 bits
+    sens_d = 0.05 + 0.9 * torch.rand(n_entries, generator=g, dtype=torch.float64)      # loss when all but 1/8 is dropped
+    quality = []
+    for i in range(n_entries):
+        row = []
+        for level, keep in forms:
+            loss_q = float(sens_q[i]) * (level / 3.0) ** 2
+            loss_d = float(sens_d[i]) * ((1.0 - keep) / 0.875) ** 1.5
+            row.append(max(0.0, (1.0 - loss_q) * (1.0 - loss_d)))
+        quality.append(row)
+    return freq, tokens, forms, quality
