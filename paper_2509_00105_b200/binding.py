@@ -17,7 +17,10 @@ CHUNK_TOKENS = 256
 GROUP = 32
 NUM_LEVELS = 4
 
-_LIB_PATH = Path(__file__).resolve().parent / "libkvh.so"
+import os
+
+# KVH_LIB names another build of the library (a measurement aid: comparing build variants)
+_LIB_PATH = Path(os.environ.get("KVH_LIB") or Path(__file__).resolve().parent / "libkvh.so")
 _lib = None
 
 

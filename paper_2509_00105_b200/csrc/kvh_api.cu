@@ -15,10 +15,6 @@
 #include "kvh_format.cuh"
 #include "kvh_host.cuh"
 
-#ifndef KVH_ENCODE_GROUPS
-#define KVH_ENCODE_GROUPS 1     // consumer groups of 256 threads in the TMA-fed encode kernel
-#endif
-
 using namespace kvh;
 
 namespace {
@@ -83,26 +79,25 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream)
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return KVH_ERR_CUDA;
-        constexpr int G = KVH_ENCODE_GROUPS;
         const size_t dyn = (size_t)kEncStages * kEncStageBytes;
         // one level for the whole launch (kvh_encode): an instance that holds only that level's code
         const int level = p.descs ? p.hint_level : p.level;
         void (*kernel)(const EncodeParams, const int, const int);
         if (p.c == 1024) {
-            kernel = level == 0 ? encode_tma_kernel<1024, G, 0> : level == 1 ? encode_tma_kernel<1024, G, 1>
-                   : level == 2 ? encode_tma_kernel<1024, G, 2> : level == 3 ? encode_tma_kernel<1024, G, 3>
-                   : encode_tma_kernel<1024, G, -1>;
+            kernel = level == 0 ? encode_tma_kernel<1024, 0> : level == 1 ? encode_tma_kernel<1024, 1>
+                   : level == 2 ? encode_tma_kernel<1024, 2> : level == 3 ? encode_tma_kernel<1024, 3>
+                   : encode_tma_kernel<1024, -1>;
         } else {
-            kernel = level == 0 ? encode_tma_kernel<0, G, 0> : level == 1 ? encode_tma_kernel<0, G, 1>
-                   : level == 2 ? encode_tma_kernel<0, G, 2> : level == 3 ? encode_tma_kernel<0, G, 3>
-                   : encode_tma_kernel<0, G, -1>;
+            kernel = level == 0 ? encode_tma_kernel<0, 0> : level == 1 ? encode_tma_kernel<0, 1>
+                   : level == 2 ? encode_tma_kernel<0, 2> : level == 3 ? encode_tma_kernel<0, 3>
+                   : encode_tma_kernel<0, -1>;
         }
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
             return KVH_ERR_CUDA;
         const char *sched_env = getenv("KVH_ENCODE_SCHED");
         const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
         const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
-        kernel<<<pgrid, 32 + G * kEncGroupThreads, dyn, st>>>(p, (int)n_chunks, sched);
+        kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, (int)n_chunks, sched);
         return launch_status();
     }
     encode_kernel<<<grid, kThreads, 0, st>>>(p);

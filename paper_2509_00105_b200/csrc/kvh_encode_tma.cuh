@@ -383,9 +383,10 @@ __device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st
 
 // sched: 0 = each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (grid = resident CTAs);
 //        1 = one CTA per tile in the grid, running CTAs pull further tiles through cluster launch control.
-// G consumer groups of 256 threads take the units in turn (unit i goes to group i % G).
-template <int C, int G, int LEVEL>
-__global__ void __launch_bounds__(32 + G * kEncGroupThreads, 1)
+// The 8 consumer warps take every unit together: a stage's full barrier is then waited on once per
+// phase, which is what lets one parity bit tell the phases apart.
+template <int C, int LEVEL>
+__global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
 encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
@@ -397,7 +398,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
     __shared__ __align__(8) uint64_t clc_bar[2];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int kProducerWarp = G * kEncGroupThreads / 32;
+    constexpr int kProducerWarp = kEncGroupThreads / 32;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kEncStages; ++s) {
@@ -518,15 +519,13 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
                 tile_id += gridDim.x;
             }
         }
-        for (int g = 0; ok && g < G; ++g) {              // one end marker per consumer group
-            ok = acquire();
-            if (ok) {
-                if (lane == 0) {
-                    info[unit % kEncStages].bits = 0;
-                    mbar_arrive(&full_bar[unit % kEncStages]);
-                }
-                ++unit;
+        if (ok) ok = acquire();
+        if (ok) {                                        // end marker
+            if (lane == 0) {
+                info[unit % kEncStages].bits = 0;
+                mbar_arrive(&full_bar[unit % kEncStages]);
             }
+            ++unit;
         }
         if (!ok && lane == 0) {
             report(p.status, KVH_ERR_TIMEOUT);
@@ -543,9 +542,8 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
         }
     } else {
         // ------------------------------ consumer warps ------------------------------
-        const int group = warp / (kEncGroupThreads / 32);
-        const int tid = threadIdx.x - group * kEncGroupThreads;
-        for (uint32_t unit = group;; unit += G) {
+        const int tid = threadIdx.x;
+        for (uint32_t unit = 0;; ++unit) {
             const int s = unit % kEncStages;
             if (!mbar_wait(&full_bar[s], (unit / kEncStages) & 1, &abort_flag)) {
                 report(p.status, KVH_ERR_TIMEOUT);

@@ -202,7 +202,7 @@ __device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, 
     if constexpr (LIN >= 0) {
         tc_consume_levels<C, LIN, LOUT>(u.e, st, c_rt, tid, eb);
     } else {
-        switch (u.bits_in * 16 + u.e.bits) {             // uniform per consumer group
+        switch (u.bits_in * 16 + u.e.bits) {             // uniform per CTA
         case 16 * 16 + 8: tc_consume_levels_call<C, 0, 1>(&u.e, st, c_rt, tid, eb); break;
         case 16 * 16 + 4: tc_consume_levels_call<C, 0, 2>(&u.e, st, c_rt, tid, eb); break;
         case 16 * 16 + 2: tc_consume_levels_call<C, 0, 3>(&u.e, st, c_rt, tid, eb); break;
