@@ -201,6 +201,8 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
     const uint32_t row_bytes = (uint32_t)c * BITS / 8;
     const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
     uint16_t *dst = r.dst;
+    const f32x2 pre01 = f2_make(Pos<BITS>::prescale(0), Pos<BITS>::prescale(1));
+    const f32x2 pre23 = f2_make(Pos<BITS>::prescale(2), Pos<BITS>::prescale(3));
     // r.count is the same for the 4 lanes of a quad (they share the row group), so the shuffles
     // below are executed by whole quads
     for (int kb = 0; kb < r.count; kb += 4) {
@@ -214,8 +216,8 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
             if (kb + j < r.count) {
                 const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
                 const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
-                const f32x2 sa = f2_make(__fmul_rn(s0, Pos<BITS>::prescale(0)), __fmul_rn(s0, Pos<BITS>::prescale(1)));
-                const f32x2 sb = f2_make(__fmul_rn(s0, Pos<BITS>::prescale(2)), __fmul_rn(s0, Pos<BITS>::prescale(3)));
+                const f32x2 ss = f2_make(s0, s0);
+                const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);      // exact: powers of two
                 const f32x2 ll = f2_make(l1, l1);
                 const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
                 f32x2 x[4];
