@@ -128,9 +128,14 @@ kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_chan
  * ceil(n_tokens/256)]: desc i describes tokens [256 i, 256 i + n_tok) and where
  * its stream goes (as laid out by kvh_plan_chunks).  A descriptor with a bad
  * level, an n_tok that does not match the context, a misaligned offset or an
- * extent beyond out_capacity is skipped and reported through *dev_status. */
+ * extent beyond out_capacity is skipped and reported through *dev_status.
+ * descs_host [host, may be NULL]: the same n_chunks descriptors in host memory.
+ * With them the call sorts the chunks by level and runs, per level, the kernel
+ * that holds only that level's code (about 1.7 times faster on mixed contexts
+ * than the one kernel that holds them all, which runs when descs_host is NULL);
+ * a chunk whose two descriptors disagree on the level is skipped and reported. */
 kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
-                             const kvh_chunk_desc *descs, int n_chunks,
+                             const kvh_chunk_desc *descs, const kvh_chunk_desc *descs_host, int n_chunks,
                              void *out, uint64_t out_capacity,
                              int32_t *dev_status, void *stream);
 

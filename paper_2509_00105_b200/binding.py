@@ -71,7 +71,7 @@ def lib() -> ctypes.CDLL:
         L.kvh_encode.restype = i32
         L.kvh_encode.argtypes = [vp, i32, i64, i32, i32, vp, u64, vp, vp]
         L.kvh_encode_chunks.restype = i32
-        L.kvh_encode_chunks.argtypes = [vp, i32, i64, i32, vp, i32, vp, u64, vp, vp]
+        L.kvh_encode_chunks.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, u64, vp, vp]
         L.kvh_decode_to_pages.restype = i32
         L.kvh_decode_to_pages.argtypes = [vp, i32, i32, vp, ctypes.POINTER(_PoolStruct), vp, vp]
         L.kvh_decode_batch.restype = i32
@@ -196,10 +196,16 @@ def encode(kv: torch.Tensor, level: int, out: torch.Tensor | None = None,
 
 
 def encode_chunks(kv: torch.Tensor, descs_dev: torch.Tensor, n_chunks: int, out: torch.Tensor,
-                  dev_status: torch.Tensor | None = None) -> None:
-    """Encode a context with one level per chunk; descs_dev is the device copy of plan_chunks()'s array."""
+                  dev_status: torch.Tensor | None = None, descs: np.ndarray | None = None) -> None:
+    """Encode a context with one level per chunk; descs_dev is the device copy of plan_chunks()'s
+    array.  Passing the host array too (`descs`) lets the library run each level's chunks through
+    the kernel specialised for that level."""
     l, N, c = _check_kv(kv)
-    _check(lib().kvh_encode_chunks(kv.data_ptr(), l, N, c, descs_dev.data_ptr(), n_chunks, out.data_ptr(),
+    host = 0
+    if descs is not None:
+        assert descs.dtype == DESC_DTYPE and len(descs) == n_chunks and descs.flags.c_contiguous
+        host = descs.ctypes.data
+    _check(lib().kvh_encode_chunks(kv.data_ptr(), l, N, c, descs_dev.data_ptr(), host, n_chunks, out.data_ptr(),
                                    out.numel(), _ptr(dev_status), _stream()), "kvh_encode_chunks")
 
 

@@ -68,37 +68,73 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
 // Encode launch: the persistent TMA-fed kernel when a 32-token tile fits a shared-memory stage,
 // otherwise one CTA per tile reading global memory directly.  KVH_ENCODE_PATH=direct forces the
 // latter and KVH_ENCODE_SCHED=static a fixed tile stride (measurement aids).
-kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream)
+template <typename Chunks>
+kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, int n_chunks, cudaStream_t st,
+                             const Chunks &chunks)
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return KVH_ERR_CUDA;
+    const size_t dyn = (size_t)kEncStages * kEncStageBytes;
+    void (*kernel)(const EncodeParams, const int, const int, const Chunks);
+    if (p.c == 1024) {
+        kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks> : level == 1 ? encode_tma_kernel<1024, 1, Chunks>
+               : level == 2 ? encode_tma_kernel<1024, 2, Chunks> : level == 3 ? encode_tma_kernel<1024, 3, Chunks>
+               : encode_tma_kernel<1024, -1, Chunks>;
+    } else {
+        kernel = level == 0 ? encode_tma_kernel<0, 0, Chunks> : level == 1 ? encode_tma_kernel<0, 1, Chunks>
+               : level == 2 ? encode_tma_kernel<0, 2, Chunks> : level == 3 ? encode_tma_kernel<0, 3, Chunks>
+               : encode_tma_kernel<0, -1, Chunks>;
+    }
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
+        return KVH_ERR_CUDA;
+    const char *sched_env = getenv("KVH_ENCODE_SCHED");
+    const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
+    const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
+    kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, n_chunks, sched, chunks);
+    return launch_status();
+}
+
+// descs_host (may be nullptr): the caller's host copy of p.descs, indexed like it.  With it the
+// chunks of each level go, as index lists in the kernel parameters, to the instance specialised for
+// that level; without it one instance that holds all levels takes the chunks in order.
+kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
+                         const kvh_chunk_desc *descs_host = nullptr)
 {
     const unsigned grid = grid_for(n_chunks, p.l);
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const char *force = getenv("KVH_ENCODE_PATH");
     if (p.c <= kEncMaxChannels && (p.n_runs > 0 || !(force && strcmp(force, "direct") == 0))) {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return KVH_ERR_CUDA;
-        const size_t dyn = (size_t)kEncStages * kEncStageBytes;
-        // one level for the whole launch (kvh_encode): an instance that holds only that level's code
         const int level = p.descs ? p.hint_level : p.level;
-        void (*kernel)(const EncodeParams, const int, const int);
-        if (p.c == 1024) {
-            kernel = level == 0 ? encode_tma_kernel<1024, 0> : level == 1 ? encode_tma_kernel<1024, 1>
-                   : level == 2 ? encode_tma_kernel<1024, 2> : level == 3 ? encode_tma_kernel<1024, 3>
-                   : encode_tma_kernel<1024, -1>;
-        } else {
-            kernel = level == 0 ? encode_tma_kernel<0, 0> : level == 1 ? encode_tma_kernel<0, 1>
-                   : level == 2 ? encode_tma_kernel<0, 2> : level == 3 ? encode_tma_kernel<0, 3>
-                   : encode_tma_kernel<0, -1>;
+        if (level >= 0 || !descs_host || !p.descs)
+            return launch_encode_tma(p, level, grid, (int)n_chunks, st, AllChunks{});
+        static thread_local ListedChunks list;           // 16 KB of parameters, filled per launch
+        EncodeParams q = p;
+        q.chunk0 = 0;
+        for (int lv = 0; lv < kNumLevels; ++lv) {
+            q.hint_level = lv;
+            int n = 0;
+            for (int64_t i = 0; i <= n_chunks; ++i) {
+                if (i < n_chunks && descs_host[p.chunk0 + i].level == lv) list.idx[n++] = (uint32_t)(p.chunk0 + i);
+                if (n == kMaxListedChunks || (i == n_chunks && n > 0)) {
+                    const kvh_status s = launch_encode_tma(q, lv, grid_for(n, p.l), n, st, list);
+                    if (s != KVH_OK) return s;
+                    n = 0;
+                }
+            }
         }
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
-            return KVH_ERR_CUDA;
-        const char *sched_env = getenv("KVH_ENCODE_SCHED");
-        const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
-        const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
-        kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, (int)n_chunks, sched);
-        return launch_status();
+        // descriptors whose level is no level at all go to the general instance, which reports and skips them
+        int n = 0;
+        for (int64_t i = 0; i < n_chunks && n < kMaxListedChunks; ++i)
+            if (descs_host[p.chunk0 + i].level < 0 || descs_host[p.chunk0 + i].level >= kNumLevels)
+                list.idx[n++] = (uint32_t)(p.chunk0 + i);
+        if (n > 0) {
+            q.hint_level = -1;
+            return launch_encode_tma(q, -1, grid_for(n, p.l), n, st, list);
+        }
+        return KVH_OK;
     }
     encode_kernel<<<grid, kThreads, 0, st>>>(p);
     return launch_status();
@@ -201,8 +237,8 @@ kvh_status kvh_encode(const void *kv, int n_layers, int64_t n_tokens, int n_chan
 }
 
 kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
-                             const kvh_chunk_desc *descs, int n_chunks, void *out, uint64_t out_capacity,
-                             int32_t *dev_status, void *stream)
+                             const kvh_chunk_desc *descs, const kvh_chunk_desc *descs_host, int n_chunks,
+                             void *out, uint64_t out_capacity, int32_t *dev_status, void *stream)
 {
     if (!kv || !out || !descs || n_tokens <= 0) return KVH_ERR_INVALID_ARG;
     const kvh_status s = check_shape(0, n_layers, n_channels);
@@ -217,7 +253,7 @@ kvh_status kvh_encode_chunks(const void *kv, int n_layers, int64_t n_tokens, int
     p.out = static_cast<uint8_t *>(out);
     p.capacity = out_capacity;
     p.status = dev_status;
-    return launch_encode(p, n_chunks, stream);
+    return launch_encode(p, n_chunks, stream, descs_host);
 }
 
 kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n_recent,
@@ -439,7 +475,7 @@ kvh_status kvh_store_host(const void *kv, int n_layers, int64_t n_tokens, int n_
         p.out = static_cast<uint8_t *>(dev_staging);
         p.capacity = staging_bytes;
         p.status = dev_status;
-        const kvh_status ls = launch_encode(p, s.count, st);
+        const kvh_status ls = launch_encode(p, s.count, st, descs_host);
         if (ls != KVH_OK) return ls;
         if (!chain(st, cp) ||
             cudaMemcpyAsync(static_cast<uint8_t *>(host_out) + s.off,

@@ -34,6 +34,18 @@ constexpr int kEncStages = 3;
 constexpr uint32_t kEncStageBytes = 2u * kTileTokens * 1024u;   // a 32-token tile at c = 1024
 constexpr int kEncMaxChannels = 1024;
 
+// Which chunks a launch covers: chunk0, chunk0 + 1, ... in order, or the ones a list names.  The
+// list travels in the kernel's parameters (no device memory), which is what lets the host hand
+// each level's chunks of a mixed context to the kernel instance specialised for that level.
+constexpr int kMaxListedChunks = 4000;
+struct AllChunks {
+    __device__ __forceinline__ int chunk(int i, int chunk0) const { return chunk0 + i; }
+};
+struct ListedChunks {
+    uint32_t idx[kMaxListedChunks];
+    __device__ __forceinline__ int chunk(int i, int) const { return (int)idx[i]; }
+};
+
 struct EncUnit {
     int32_t bits;          // 16, 8, 4, 2; 0 marks the end of the CTA's work
     int32_t kv;            // 0 K, 1 V
@@ -385,9 +397,9 @@ __device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st
 //        1 = one CTA per tile in the grid, running CTAs pull further tiles through cluster launch control.
 // The 8 consumer warps take every unit together: a stage's full barrier is then waited on once per
 // phase, which is what lets one parity bit tell the phases apart.
-template <int C, int LEVEL>
+template <int C, int LEVEL, typename Chunks>
 __global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
-encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
+encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, const Chunks chunks)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kEncStages];
@@ -431,7 +443,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched)
             const int64_t plane_id = tile_id / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
-            const int chunk = p.chunk0 + (int)((plane_id >> 1) / p.l);
+            const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), p.chunk0);
             const int64_t tok0 = (int64_t)chunk * kChunkTokens;
             const int n_expect = (int)min((int64_t)kChunkTokens, p.N - tok0);
             kvh_chunk_desc d;

@@ -179,6 +179,10 @@ def test_batched_mixed_level_decode_into_shared_pool(kvh):
         out = torch.full((total,), 0xCD, dtype=torch.uint8, device="cuda")
         kvh.encode_chunks(kv, kvh.descs_to_tensor(local, "cuda"), len(levels), out, status)
         assert np.array_equal(out.cpu().numpy(), want)
+        # the same with the host copy of the descriptors: one specialised launch per level
+        out.fill_(0xCD)
+        kvh.encode_chunks(kv, kvh.descs_to_tensor(local, "cuda"), len(levels), out, status, descs=local)
+        assert np.array_equal(out.cpu().numpy(), want)
         npg = workloads.n_pages(N)
         ids = perm[pt_base:pt_base + npg]
         ntoks, lv, _ = oracle.chunk_plan(N, levels, l, c)
@@ -312,3 +316,33 @@ def test_encode_rounds_ties_like_the_oracle(kvh, l, c, N, level):
     want, _ = oracle.encode_context(kv_np, level)
     got, _ = kvh.encode(from_np16(kv_np), level)
     assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_mixed_level_encode_with_host_descriptors(kvh):
+    """c = 1024, many chunks, every level: per-level launches over chunk lists must produce the same
+    stream as the oracle; a chunk whose host and device descriptors disagree is skipped and reported."""
+    l, c, N = 2, 1024, 256 * 37 + 100
+    kv = workloads.make_kv(l, N, c, seed=91, device="cuda")
+    levels = workloads.chunk_levels(workloads.n_chunks(N), 4, seed=92)
+    assert set(levels) == {0, 1, 2, 3}
+    want, offsets = oracle.encode_context(to_np16(kv), levels)
+    descs, total = kvh.plan_chunks(l, c, N, levels)
+    out = torch.full((total,), 0xCD, dtype=torch.uint8, device="cuda")
+    status = new_status()
+    kvh.encode_chunks(kv, kvh.descs_to_tensor(descs, "cuda"), len(descs), out, status, descs=descs)
+    assert status.item() == 0
+    assert np.array_equal(out.cpu().numpy(), want)
+    # chunk 5: the host says another level than the device; chunk 7: the host names no level at all
+    lie = descs.copy()
+    lie["level"][5] = (levels[5] + 1) % 4
+    lie["level"][7] = 9
+    out.fill_(0xCD)
+    kvh.encode_chunks(kv, kvh.descs_to_tensor(descs, "cuda"), len(descs), out, status, descs=lie)
+    assert status.item() == 2
+    o = out.cpu().numpy()
+    for i in range(len(descs)):
+        a, b = offsets[i], offsets[i + 1]
+        if i == 5:
+            assert np.all(o[a:b] == 0xCD)
+        else:                                            # chunk 7 is encoded by the general kernel from its device descriptor
+            assert np.array_equal(o[a:b], want[a:b])

@@ -102,7 +102,7 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(kvh):
     assert L.kvh_encode(a + 8, 1, 256, 32, 0, a, 1 << 20, None, None) == 4
     assert L.kvh_encode(a, 1, 256, 32, 0, a + 64, 1 << 20, None, None) == 4
     assert L.kvh_encode(a, 1, 256, 32, 0, a, 100, None, None) == 5
-    assert L.kvh_encode_chunks(a, 1, 600, 32, a, 2, a, 1 << 20, None, None) == 3      # 600 tokens = 3 chunks
+    assert L.kvh_encode_chunks(a, 1, 600, 32, a, None, 2, a, 1 << 20, None, None) == 3      # 600 tokens = 3 chunks
     pool = kvh.binding._PoolStruct(a, 2 * 8 * 16 * 32, 8 * 16 * 32, 16 * 32, 8, 16, 1, 32)
     assert L.kvh_decode_to_pages(None, 0, 16, a, ctypes.byref(pool), None, None) == 1
     assert L.kvh_decode_to_pages(a, 4, 16, a, ctypes.byref(pool), None, None) == 2
