@@ -200,9 +200,13 @@ kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes,
  * chunks that break a rule are skipped and reported through *dev_status (pt_off is not used).
  * level_in / level_out: when every chunk goes from one level to one other level, pass them and a
  * kernel specialised for the pair runs (chunks with other levels are skipped and reported);
- * pass -1 / -1 for any mix.  The two buffers must not overlap.  n_channels <= 1024. */
+ * pass -1 / -1 for any mix.  in_descs_host / out_descs_host [host, n_chunks each, may both be
+ * NULL]: host copies of the two arrays; with them a mix is sorted by pair of levels on the host
+ * and every pair runs through its specialised kernel (as kvh_encode_chunks does per level).  The
+ * two stream buffers must not overlap.  n_channels <= 1024. */
 kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, const kvh_chunk_desc *in_descs,
                          void *out_streams, uint64_t out_capacity, const kvh_chunk_desc *out_descs,
+                         const kvh_chunk_desc *in_descs_host, const kvh_chunk_desc *out_descs_host,
                          int n_chunks, int n_layers, int n_channels, int level_in, int level_out,
                          int32_t *dev_status, void *stream);
 

@@ -86,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.kvh_encode_kept.restype = i32
         L.kvh_encode_kept.argtypes = [vp, i32, i64, i32, vp, i32, vp, i32, i32, vp, u64, vp, vp]
         L.kvh_transcode.restype = i32
-        L.kvh_transcode.argtypes = [vp, u64, vp, vp, u64, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.kvh_transcode.argtypes = [vp, u64, vp, vp, u64, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
         L.kvh_policy_assign.restype = i32
         L.kvh_policy_assign.argtypes = [vp, vp, vp, i32, vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_double)]
         L.kvh_policy_assign_tiers.restype = i32
@@ -317,14 +317,21 @@ def encode_kept(kv: torch.Tensor, runs, descs_dev: torch.Tensor | None, n_chunks
 
 def transcode(in_streams: torch.Tensor, in_descs_dev: torch.Tensor, out_streams: torch.Tensor,
               out_descs_dev: torch.Tensor, n_chunks: int, n_layers: int, n_channels: int,
-              level_in: int = -1, level_out: int = -1, dev_status: torch.Tensor | None = None) -> None:
+              level_in: int = -1, level_out: int = -1, dev_status: torch.Tensor | None = None,
+              in_descs: np.ndarray | None = None, out_descs: np.ndarray | None = None) -> None:
     """Re-encode stored chunks at a coarser level on the device.  level_in/level_out name the one
-    pair of levels all chunks share, or -1/-1 for a mix taken from the descriptors."""
+    pair of levels all chunks share, or -1/-1 for a mix taken from the descriptors; for a mix the
+    host arrays (in_descs, out_descs) let every pair of levels run through its own kernel."""
     assert in_streams.is_cuda and in_streams.dtype == torch.uint8
     assert out_streams.is_cuda and out_streams.dtype == torch.uint8
     assert in_descs_dev.numel() >= 24 * n_chunks and out_descs_dev.numel() >= 24 * n_chunks
+    hi = ho = 0
+    if in_descs is not None and out_descs is not None:
+        assert in_descs.dtype == DESC_DTYPE and out_descs.dtype == DESC_DTYPE
+        assert len(in_descs) == len(out_descs) == n_chunks and in_descs.flags.c_contiguous and out_descs.flags.c_contiguous
+        hi, ho = in_descs.ctypes.data, out_descs.ctypes.data
     _check(lib().kvh_transcode(in_streams.data_ptr(), in_streams.numel(), in_descs_dev.data_ptr(),
-                               out_streams.data_ptr(), out_streams.numel(), out_descs_dev.data_ptr(), n_chunks,
+                               out_streams.data_ptr(), out_streams.numel(), out_descs_dev.data_ptr(), hi, ho, n_chunks,
                                n_layers, n_channels, level_in, level_out, _ptr(dev_status), _stream()),
            "kvh_transcode")
 

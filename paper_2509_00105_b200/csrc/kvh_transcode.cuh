@@ -214,9 +214,9 @@ __device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, 
 }
 
 // sched as in the encode kernel.  One CTA per SM: 8 consumer warps and a producer warp.
-template <int C, int LIN, int LOUT>
+template <int C, int LIN, int LOUT, typename Chunks>
 __global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
-transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sched)
+transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sched, const Chunks chunks)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kEncStages];
@@ -264,7 +264,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
             const int64_t plane_id = tile_id / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
-            const int chunk = (int)((plane_id >> 1) / p.l);
+            const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), 0);
             if (chunk != cur_chunk) {
                 cur_chunk = chunk;
                 di = p.in_descs[chunk];

@@ -38,6 +38,14 @@ def run_case(kvh, l, c, N, levels_in, levels_out, hint):
     assert status.item() == 0
     assert np.array_equal(g[:total], want)
     assert np.all(g[total:] == 0xAB)
+    if hint == (-1, -1):                                 # with the host descriptors: one launch per pair of levels
+        out.fill_(0xAB)
+        kvh.transcode(torch.from_numpy(src).cuda(), kvh.descs_to_tensor(din, "cuda"), out[:total],
+                      kvh.descs_to_tensor(dout, "cuda"), len(din), l, c, -1, -1, dev_status=status,
+                      in_descs=din, out_descs=dout)
+        g = out.cpu().numpy()
+        assert status.item() == 0
+        assert np.array_equal(g[:total], want) and np.all(g[total:] == 0xAB)
 
 
 @pytest.mark.parametrize("l,c,N", [(1, 1024, 300), (2, 256, 257), (1, 32, 33), (1, 96, 700), (2, 1024, 64)])
@@ -75,6 +83,14 @@ def test_transcode_skips_and_reports_chunks_that_break_a_rule(kvh):
         o = out.cpu().numpy()
         assert status.item() == expect
         assert np.array_equal(o[:half], want[:half]) and np.all(o[half:] == 0xEE)   # chunk 0 fine, chunk 1 untouched
+        if hint == (-1, -1):                             # the same when the host knows the descriptors
+            out.fill_(0xEE)
+            status.zero_()
+            kvh.transcode(src, kvh.descs_to_tensor(a, "cuda"), out[:capacity or total + room], kvh.descs_to_tensor(b, "cuda"),
+                          2, l, c, -1, -1, dev_status=status, in_descs=a, out_descs=b)
+            o = out.cpu().numpy()
+            assert status.item() == expect
+            assert np.array_equal(o[:half], want[:half]) and np.all(o[half:] == 0xEE)
 
     nop = lambda d: None
     run(nop, lambda d: d["level"].__setitem__(1, 1), 2)              # not coarser
