@@ -264,10 +264,8 @@ __device__ __forceinline__ void enc_unrotate(uint32_t (&p)[4][W], int rot)
         for (int w = 0; w < W; ++w) p[k][w] = r2 ? q[(k + 2) & 3][w] : q[k][w];
 }
 
-// One group: range, metadata word, codes.  x[j] is the 16-byte piece number (j + rot) & 3 of the
-// group's 64 bytes (ROTATED), or simply piece j.
-template <int BITS, bool ROTATED = true>
-__device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32_t *meta_out, uint8_t *codes_out)
+// Metadata word (min | max << 16) of one group given as four 16-byte pieces, in any order.
+__device__ __forceinline__ uint32_t enc_range_v(const uint4 (&x)[4])
 {
     uint32_t mn = bmin2(bmin2(x[0].x, x[0].y), bmin2(x[0].z, x[0].w));
     uint32_t mx = bmax2(bmax2(x[0].x, x[0].y), bmax2(x[0].z, x[0].w));
@@ -278,7 +276,15 @@ __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32
     }
     mn = bmin2(mn, swap_halves(mn));
     mx = bmax2(mx, swap_halves(mx));
-    const uint32_t m = __byte_perm(mn, mx, 0x5410);
+    return __byte_perm(mn, mx, 0x5410);
+}
+
+// One group with its metadata word m known: store m and the codes.  x[j] is the 16-byte piece
+// number (j + rot) & 3 of the group's 64 bytes (ROTATED), or simply piece j.
+template <int BITS, bool ROTATED = true>
+__device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32_t m, uint32_t *meta_out,
+                                            uint8_t *codes_out)
+{
     *meta_out = m;
     float lo, inv;
     encode_params<BITS>(m, lo, inv);
@@ -349,7 +355,7 @@ __device__ __forceinline__ void enc_consume_v(const uint8_t *st, int c_rt, int t
 #pragma unroll
         for (int k = 0; k < U; ++k) {
             const int g = g0 + k * kEncGroupThreads;
-            if (g < ngroups) enc_group_v<BITS>(x[k], rot, meta + g, codes + (size_t)g * (4 * BITS));
+            if (g < ngroups) enc_group_v<BITS>(x[k], rot, enc_range_v(x[k]), meta + g, codes + (size_t)g * (4 * BITS));
         }
     }
 }

@@ -9,9 +9,11 @@
 //
 // Structure: the encode kernel's pipeline (3 shared-memory stages fed by 1-D bulk copies, tiles
 // handed out through cluster launch control, 8 consumer warps) with the decode kernel's unpacking
-// in front.  A K thread dequantises the 32 rows of its 4 channels into packed bf16 registers and
-// continues exactly like the encoder; a V thread dequantises one whole 32-channel group.  A
-// level-0 source is the encoder itself reading the chunk's raw rows.
+// in front.  A level-0 source is the encoder itself reading the chunk's raw rows.  From a
+// quantised source the new range of every group follows from its old metadata (tc_new_meta), so a
+// K thread walks the rows of its 4 channels and a V thread its groups, one at a time: dequantise,
+// round to bf16, quantise again, store.  Such instances need few registers and small stages and
+// run two CTAs per SM.
 #pragma once
 
 #include "kvh_async.cuh"
@@ -65,21 +67,17 @@ __device__ __forceinline__ void spread4(const uint8_t *src, f32x2 (&x)[2])
     x[1] = f2_sub(f2_from_bits(m[2], m[3]), bias);
 }
 
-// Decode parameters of a thread's 4 K channels (metadata words in shared memory), with the scale
-// pre-multiplied by 2^-position as the decode kernel does.
+// A decoded group needs no second look to know its range.  Its smallest element had code 0 and its
+// largest code qmax (the quantiser maps min to 0 and max to qmax whatever the rounding), and
+// decoding is monotone, so the decoded values span exactly [xhat(0), xhat(qmax)] and the metadata
+// word of the re-encoded group follows from the old one alone.  That makes every element
+// independent: the kernel streams rows instead of holding a tile in registers.
 template <int BIN>
-__device__ __forceinline__ void tc_params_k(const uint8_t *meta, int cq, f32x2 (&lo)[2], f32x2 (&sc)[2])
+__device__ __forceinline__ uint32_t tc_new_meta(uint32_t m, float &lo, float &scale)
 {
-    const uint4 w4 = *reinterpret_cast<const uint4 *>(meta + 16 * (size_t)cq);
-    const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-    float l1[4], s1[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        decode_params<BIN>(w[i], l1[i], s1[i]);
-        s1[i] = __fmul_rn(s1[i], Pos<BIN>::prescale(i));
-    }
-    lo[0] = f2_make(l1[0], l1[1]); lo[1] = f2_make(l1[2], l1[3]);
-    sc[0] = f2_make(s1[0], s1[1]); sc[1] = f2_make(s1[2], s1[3]);
+    decode_params<BIN>(m, lo, scale);
+    const float qmax = (float)((1 << BIN) - 1);
+    return pack_bf16x2_rn(__fmaf_rn(0.0f, scale, lo), __fmaf_rn(qmax, scale, lo));      // xhat(0) | xhat(qmax) << 16
 }
 
 // One dequantised K row of a 4-channel column as two packed bf16 pairs.
@@ -95,36 +93,46 @@ __device__ __forceinline__ uint2 tc_row_k(const uint8_t *codes, const f32x2 (&lo
                       pack_bf16x2_rn(__uint_as_float(c2), __uint_as_float(d)));
 }
 
+// K: a thread owns 4 channels and walks the tile's rows (any number of them).
 template <int BIN, int BOUT, int C>
 __device__ __forceinline__ void tc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
-                                             int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+                                             int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int c = C ? C : c_rt;
-    const int C4 = c >> 2;
-    const bool active = tid < C4;
-    const int cq = active ? tid : 0;
-    f32x2 lo[2], sc[2];
-    tc_params_k<BIN>(st + tc_meta_off(c), cq, lo, sc);
-    const uint32_t row_bytes = (uint32_t)c * BIN / 8;
-    const uint8_t *src = st + (size_t)cq * BIN / 2;       // 4 codes = BIN / 2 bytes
-    uint2 x[kTileTokens];
-#pragma unroll
-    for (int t = 0; t < kTileTokens; ++t) x[t] = tc_row_k<BIN>(src + (size_t)t * row_bytes, lo, sc);
-    enc_release(empty_bar);
-    if (active) enc_process_k<BOUT, C>(x, c_rt, cq, tile, meta_sec, codes_sec);
-}
-
-template <int BIN, int BOUT>
-__device__ __noinline__ void tc_consume_k_short(const uint8_t *st, int c, int tid, uint64_t *empty_bar,
-                                                int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
-{
     if (tid < (c >> 2)) {
-        f32x2 lo[2], sc[2];
-        tc_params_k<BIN>(st + tc_meta_off(c), tid, lo, sc);
-        const uint32_t row_bytes = (uint32_t)c * BIN / 8;
-        const uint8_t *src = st + (size_t)tid * BIN / 2;
-        enc_k_short<BOUT>([&](int t) { return tc_row_k<BIN>(src + (size_t)t * row_bytes, lo, sc); },
-                          c, tid, nt, tile, meta_sec, codes_sec);
+        const int cq = tid;
+        const uint4 w4 = *reinterpret_cast<const uint4 *>(st + tc_meta_off(c) + 16 * (size_t)cq);
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        float l1[4], s1[4], lo_new[4], inv[4];
+        uint32_t m[4], mask[4];
+        bool all_quantised = true;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            m[i] = tc_new_meta<BIN>(w[i], l1[i], s1[i]);
+            s1[i] = __fmul_rn(s1[i], Pos<BIN>::prescale(i));
+            encode_params<BOUT>(m[i], lo_new[i], inv[i]);
+            mask[i] = inv[i] != 0.0f ? 0xffffffffu : 0u;
+            all_quantised = all_quantised && inv[i] != 0.0f;
+        }
+        *reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)) = make_uint4(m[0], m[1], m[2], m[3]);
+        const f32x2 lo[2] = {f2_make(l1[0], l1[1]), f2_make(l1[2], l1[3])};
+        const f32x2 sc[2] = {f2_make(s1[0], s1[1]), f2_make(s1[2], s1[3])};
+        const f32x2 lo_a = f2_make(lo_new[0], lo_new[1]), lo_b = f2_make(lo_new[2], lo_new[3]);
+        const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
+        const uint32_t in_bytes = (uint32_t)c * BIN / 8, out_bytes = (uint32_t)c * BOUT / 8;
+        const uint8_t *src = st + (size_t)cq * BIN / 2;   // 4 codes = BIN / 2 bytes
+        uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BOUT / 8;
+        if (all_quantised) {
+#pragma unroll 8
+            for (int t = 0; t < nt; ++t)
+                enc_store_row_k<BOUT, false>(tc_row_k<BIN>(src + (size_t)t * in_bytes, lo, sc), lo_a, lo_b, inv_a, inv_b,
+                                             mask, out + (size_t)t * out_bytes);
+        } else {
+#pragma unroll 1
+            for (int t = 0; t < nt; ++t)
+                enc_store_row_k<BOUT, true>(tc_row_k<BIN>(src + (size_t)t * in_bytes, lo, sc), lo_a, lo_b, inv_a, inv_b,
+                                            mask, out + (size_t)t * out_bytes);
+        }
     }
     enc_release(empty_bar);
 }
@@ -141,37 +149,26 @@ __device__ __forceinline__ void tc_consume_v(const uint8_t *st, int c_rt, int ti
     const size_t g_first = (size_t)tile * kTileTokens * gpr;
     uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec) + g_first;
     uint8_t *codes = codes_sec + g_first * (4 * BOUT);
-    constexpr int U = 2;
-    const int iters = (ngroups + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);  // the same for every thread
-    for (int it = 0; it < iters; ++it) {
-        const int g0 = it * kEncGroupThreads * U + tid;
-        uint4 x[U][4];
+    const f32x2 pre01 = f2_make(Pos<BIN>::prescale(0), Pos<BIN>::prescale(1));
+    const f32x2 pre23 = f2_make(Pos<BIN>::prescale(2), Pos<BIN>::prescale(3));
+#pragma unroll 2
+    for (int g = tid; g < ngroups; g += kEncGroupThreads) {
+        float l1, s0;
+        const uint32_t m = tc_new_meta<BIN>(meta_in[g], l1, s0);
+        const f32x2 ss = f2_make(s0, s0), ll = f2_make(l1, l1);
+        const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);          // exact: powers of two
+        const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+        const uint8_t *src = st + (size_t)g * (4 * BIN);  // 32 codes = 4 * BIN bytes
+        uint4 x[4];
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const int g = g0 + k * kEncGroupThreads;
-            if (g < ngroups) {
-                float l1, s0;
-                decode_params<BIN>(meta_in[g], l1, s0);
-                const f32x2 sa = f2_make(__fmul_rn(s0, Pos<BIN>::prescale(0)), __fmul_rn(s0, Pos<BIN>::prescale(1)));
-                const f32x2 sb = f2_make(__fmul_rn(s0, Pos<BIN>::prescale(2)), __fmul_rn(s0, Pos<BIN>::prescale(3)));
-                const f32x2 ll = f2_make(l1, l1);
-                const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
-                const uint8_t *src = st + (size_t)g * (4 * BIN);       // 32 codes = 4 * BIN bytes
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    f32x2 q[4];
-                    spread8<BIN>(src + j * BIN, q);
-                    x[k][j] = fma_pack8(q, sc, lo);
-                }
-            }
+        for (int j = 0; j < 4; ++j) {
+            f32x2 q[4];
+            spread8<BIN>(src + j * BIN, q);
+            x[j] = fma_pack8(q, sc, lo);
         }
-        if (it == iters - 1) enc_release(empty_bar);
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const int g = g0 + k * kEncGroupThreads;
-            if (g < ngroups) enc_group_v<BOUT, false>(x[k], 0, meta + g, codes + (size_t)g * (4 * BOUT));
-        }
+        enc_group_v<BOUT, false>(x, 0, m, meta + g, codes + (size_t)g * (4 * BOUT));
     }
+    enc_release(empty_bar);
 }
 
 // One unit with both levels known at compile time (LOUT > LIN).
@@ -184,8 +181,7 @@ __device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_
     } else {
         constexpr int BIN = 16 >> LIN, BOUT = 16 >> LOUT;
         if (u.kv) tc_consume_v<BIN, BOUT, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
-        else if (u.nt == kTileTokens) tc_consume_k<BIN, BOUT, C>(st, c_rt, tid, eb, u.tile, u.meta, u.codes);
-        else tc_consume_k_short<BIN, BOUT>(st, C ? C : c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        else tc_consume_k<BIN, BOUT, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
     }
 }
 template <int C, int LIN, int LOUT>
@@ -214,8 +210,13 @@ __device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, 
 }
 
 // sched as in the encode kernel.  One CTA per SM: 8 consumer warps and a producer warp.
+// Bytes of a stage: a raw tile (64 KiB at c = 1024) when the source may be level 0, else codes of at
+// most 8 bits plus metadata (36 KiB), which leaves room for two CTAs per SM.
+template <int LIN>
+__host__ __device__ constexpr uint32_t tc_stage_bytes() { return LIN >= 1 ? 36u * 1024u : kEncStageBytes; }
+
 template <int C, int LIN, int LOUT, typename Chunks>
-__global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
+__global__ void __launch_bounds__(32 + kEncGroupThreads, LIN >= 1 ? 2 : 1)
 transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sched, const Chunks chunks)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
@@ -303,7 +304,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
                 u.e.codes_padded = (uint32_t)Lo.kcodes;
                 u.e.meta = lay_out + Lo.meta_off(kv);
                 u.e.codes = lay_out + Lo.codes_off(kv);
-                uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+                uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
                 const uint8_t *codes_in = lay_in + Li.codes_off(kv);
                 if (di.level == 0) {
                     const uint32_t bytes = 2u * (uint32_t)nt * (uint32_t)p.c;
@@ -387,7 +388,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
             }
             const TcUnit u = info[s];
             if (u.e.bits == 0) break;
-            const uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+            const uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
             if (u.e.last && tid < KVH_SECTION_ALIGN) {   // the plane's last tile clears the padding
                 if (u.e.codes_payload + tid < u.e.codes_padded) u.e.codes[u.e.codes_payload + tid] = 0;
                 if (u.e.meta_payload + tid < u.e.meta_padded) u.e.meta[u.e.meta_payload + tid] = 0;
