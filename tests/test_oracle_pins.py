@@ -570,3 +570,25 @@ def test_transcoding_error_and_range_properties():
     bound = r[:, None, :] * (0.5 / 255 + 0.5 / 3) + 2.0 ** -7 * np.abs(k).max(1)[:, None, :]
     assert np.all(np.abs(k3 - k) <= bound)
     assert np.abs(v3 - x).mean() > np.abs(v1 - x).mean()  # and it is the coarser of the two
+
+
+@pytest.mark.parametrize("level", [1, 2, 3])
+def test_decoded_group_spans_exactly_the_decodings_of_code_0_and_code_qmax(level):
+    """What the transcoding kernel relies on: a group's smallest element has code 0, its largest
+    code qmax, and decoding is monotone, so min and max of the decoded group (in the format's
+    order, -0 below +0) are dequantize(0) and dequantize(qmax) of the old metadata."""
+    bits = 16 >> level
+    qmax = (1 << bits) - 1
+    rng = np.random.default_rng(level)
+    groups = [_rand_kv(1, 32, 32, 40 + level)[0, 0, :, i] for i in range(32)]
+    groups += [rng.integers(0, 0x80, 32).astype(np.uint16),                       # subnormals: stored flat
+               rng.choice(np.array([0x0000, 0x8000], dtype=np.uint16), 32),       # signed zeros
+               rng.choice(np.array([0x7F00, 0xFF00], dtype=np.uint16), 32),       # range overflows
+               np.full(32, 0xC000, dtype=np.uint16),
+               (rng.integers(0, 200, 32).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)]
+    for g in groups:
+        g = np.ascontiguousarray(g, dtype=np.uint16)
+        mn, mx = oracle.group_range(g)
+        dec = np.array([oracle.dequantize(oracle.quantize(int(x), mn, mx, bits), mn, mx, bits) for x in g], dtype=np.uint16)
+        dmn, dmx = oracle.group_range(dec)
+        assert (dmn, dmx) == (oracle.dequantize(0, mn, mx, bits), oracle.dequantize(qmax, mn, mx, bits))
