@@ -148,3 +148,36 @@ def test_kept_runs_match_the_oracle(kvh):
         kvh.keep_sinks_and_recent(0, 1, 1)
     with pytest.raises(kvh.KvhError):
         kvh.keep_sinks_and_recent(10, -1, 1)
+
+
+def test_launches_too_large_for_a_grid_and_new_entry_points_reject_before_any_cuda_call(kvh):
+    L = kvh.lib()
+    buf = (ctypes.c_uint8 * 4096)()
+    a = (ctypes.addressof(buf) + 127) & ~127
+    # one CTA per (chunk, layer, K|V, tile): 2^27 chunks x 80 layers x 16 does not fit a grid
+    wide = kvh.binding._PoolStruct(a, 2 * 8 * 16 * 32, 8 * 16 * 32, 16 * 32, 8, 16, 80, 32)
+    assert L.kvh_decode_batch(a, 1 << 40, a, 1 << 27, a, 1 << 31, ctypes.byref(wide), None, None) == 3
+    assert L.kvh_encode(a, 80, (1 << 27) * 256, 32, 3, a, 1 << 60, None, None) == 3
+    assert L.kvh_transcode(a, 1 << 40, a, a, 1 << 40, a, None, None, 1 << 27, 80, 32, -1, -1, None, None) == 3
+    # transcode: levels, shapes, alignment
+    assert L.kvh_transcode(None, 4096, a, a, 4096, a, None, None, 1, 1, 32, -1, -1, None, None) == 1
+    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 32, 2, 1, None, None) == 2
+    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 32, 1, -1, None, None) == 2
+    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 2048, 0, 1, None, None) == 3
+    assert L.kvh_transcode(a + 64, 4096, a, a, 4096, a, None, None, 1, 1, 32, 0, 1, None, None) == 4
+    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 0, 1, 32, 0, 1, None, None) == 0      # nothing to do
+    # token dropping: runs
+    runs = (ctypes.c_int64 * 4)(0, 10, 5, 10)                                     # overlapping
+    assert L.kvh_encode_kept(a, 1, 100, 32, runs, 2, a, 1, -1, a, 1 << 20, None, None) == 1
+    runs = (ctypes.c_int64 * 2)(0, 10)
+    assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 1, -1, a, 1 << 20, None, None) == 1   # no descriptors, no level
+    assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 2, 1, a, 1 << 20, None, None) == 3    # 10 kept tokens = 1 chunk
+    assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 1, 1, a, 64, None, None) == 5
+    assert L.kvh_encode_kept(a, 1, 100, 2048, runs, 1, None, 1, 1, a, 1 << 20, None, None) == 3
+    # policy: arguments
+    assert L.kvh_policy_assign(None, a, a, 1, a, a, None, None) == 1
+    tier = np.array([(1.0, 0.0, 100)], dtype=kvh.TIER_DTYPE)                      # bandwidth must be positive
+    freq = np.array([1.0]); opts = np.array([(10, 1.0)], dtype=kvh.OPTION_DTYPE); begin = np.array([0, 1], dtype=np.int32)
+    choice = np.zeros(1, dtype=np.int32)
+    assert L.kvh_policy_assign(freq.ctypes.data, opts.ctypes.data, begin.ctypes.data, 1, tier.ctypes.data,
+                               choice.ctypes.data, None, None) == 1
