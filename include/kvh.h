@@ -164,7 +164,8 @@ kvh_status kvh_keep_sinks_and_recent(int64_t n_tokens, int64_t n_sink, int64_t n
  * chunk is stored at this one level: descs may then be NULL (chunk i lands at i *
  * kvh_level_bytes(level, ..., 256), as with kvh_encode), a kernel holding only that level's code
  * runs, and a descriptor of another level is skipped and reported; level = -1 takes a level per
- * chunk from descs.  Everything else as for kvh_encode_chunks.  n_channels must not exceed 1024
+ * chunk from descs.  Everything else as for kvh_encode_chunks.  Rows wider than 1024 channels must
+ * be divisible into equal blocks of at most 1024 channels that are multiples of 128
  * (KVH_ERR_BAD_SHAPE otherwise). */
 kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n_channels,
                            const kvh_token_run *runs, int n_runs,

@@ -82,6 +82,10 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
         kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks> : level == 1 ? encode_tma_kernel<1024, 1, Chunks>
                : level == 2 ? encode_tma_kernel<1024, 2, Chunks> : level == 3 ? encode_tma_kernel<1024, 3, Chunks>
                : encode_tma_kernel<1024, -1, Chunks>;
+    } else if (p.bw == 1024) {                           // wider rows in blocks of 1024 channels
+        kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks, true> : level == 1 ? encode_tma_kernel<1024, 1, Chunks, true>
+               : level == 2 ? encode_tma_kernel<1024, 2, Chunks, true> : level == 3 ? encode_tma_kernel<1024, 3, Chunks, true>
+               : encode_tma_kernel<1024, -1, Chunks, true>;
     } else {
         kernel = level == 0 ? encode_tma_kernel<0, 0, Chunks> : level == 1 ? encode_tma_kernel<0, 1, Chunks>
                : level == 2 ? encode_tma_kernel<0, 2, Chunks> : level == 3 ? encode_tma_kernel<0, 3, Chunks>
@@ -106,12 +110,20 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const char *force = getenv("KVH_ENCODE_PATH");
-    if (p.c <= kEncMaxChannels && (p.n_runs > 0 || !(force && strcmp(force, "direct") == 0))) {
+    const int bw = block_width(p.c);
+    if (bw > 0 && (p.n_runs > 0 || !(force && strcmp(force, "direct") == 0))) {
+        EncodeParams q = p;
+        q.bw = bw;
+        q.n_blocks = p.c / bw;
+        auto tiles = [&](int64_t chunks) -> unsigned {   // one CTA per tile and column block; 0 if too many
+            const int64_t g = (int64_t)grid_for(chunks, p.l) * q.n_blocks;
+            return (grid_for(chunks, p.l) == 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;
+        };
+        if (tiles(n_chunks) == 0) return KVH_ERR_BAD_SHAPE;
         const int level = p.descs ? p.hint_level : p.level;
         if (level >= 0 || !descs_host || !p.descs)
-            return launch_encode_tma(p, level, grid, (int)n_chunks, st, AllChunks{});
+            return launch_encode_tma(q, level, tiles(n_chunks), (int)n_chunks, st, AllChunks{});
         static thread_local ListedChunks list;           // 16 KB of parameters, filled per launch
-        EncodeParams q = p;
         q.chunk0 = 0;
         for (int lv = 0; lv < kNumLevels; ++lv) {
             q.hint_level = lv;
@@ -119,7 +131,7 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
             for (int64_t i = 0; i <= n_chunks; ++i) {
                 if (i < n_chunks && descs_host[p.chunk0 + i].level == lv) list.idx[n++] = (uint32_t)(p.chunk0 + i);
                 if (n == kMaxListedChunks || (i == n_chunks && n > 0)) {
-                    const kvh_status s = launch_encode_tma(q, lv, grid_for(n, p.l), n, st, list);
+                    const kvh_status s = launch_encode_tma(q, lv, tiles(n), n, st, list);
                     if (s != KVH_OK) return s;
                     n = 0;
                 }
@@ -132,7 +144,7 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
                 list.idx[n++] = (uint32_t)(p.chunk0 + i);
         if (n > 0) {
             q.hint_level = -1;
-            return launch_encode_tma(q, -1, grid_for(n, p.l), n, st, list);
+            return launch_encode_tma(q, -1, tiles(n), n, st, list);
         }
         return KVH_OK;
     }
@@ -283,7 +295,7 @@ kvh_status kvh_encode_kept(const void *kv, int n_layers, int64_t n_tokens, int n
         return KVH_ERR_INVALID_ARG;
     const kvh_status s = check_shape(level < 0 ? 0 : level, n_layers, n_channels);
     if (s != KVH_OK) return s;
-    if (n_channels > kEncMaxChannels) return KVH_ERR_BAD_SHAPE;       // the gather is the TMA kernel's
+    if (block_width(n_channels) == 0) return KVH_ERR_BAD_SHAPE;       // the gather is the TMA-fed kernel's
     if (!aligned(kv, 16) || !aligned(out, KVH_SECTION_ALIGN) || !aligned(descs, 8)) return KVH_ERR_MISALIGNED;
     EncodeParams p{};
     int64_t end = 0, kept = 0;

@@ -36,6 +36,7 @@ struct EncodeParams {
     const kvh_chunk_desc *descs;   // device array indexed by chunk, or nullptr for one level throughout
     int32_t chunk0;                // first chunk this launch covers
     int32_t level;                 // used when descs == nullptr
+    int32_t bw, n_blocks;          // TMA-fed kernel: channels per column block (c when c <= 1024) and blocks per row
     int32_t hint_level;            // >= 0: every chunk has this level (an instance holding only its code runs); -1: any
     uint64_t full_chunk_bytes;     // kvh_level_bytes(level, l, c, 256), same case
     uint8_t *out;

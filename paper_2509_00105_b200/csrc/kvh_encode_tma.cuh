@@ -55,7 +55,24 @@ struct EncUnit {
     uint32_t meta_payload, meta_padded, codes_payload, codes_padded;
     uint8_t *meta;         // the plane's metadata section in the stream
     uint8_t *codes;        // the plane's code section
+    int32_t col0;          // first channel of the tile's column block (0 unless rows are wider than a stage holds)
+    int32_t cw;            // channels per row of the block = per stage row
 };
+
+// Rows wider than 1024 channels are cut into column blocks of equal width (a divisor of c that is a
+// multiple of 128); a tile is then 32 tokens of one block.  In the stage its rows are cw channels
+// wide and packed; in the plane (source and stream) rows are cf channels wide and the block starts
+// at channel col0.  With the channel count compiled in, all three are constants.
+struct RowGeom {
+    int cw, cf, col0;
+};
+template <int C, bool WIDE = false>
+__device__ __forceinline__ RowGeom row_geom(int cw, int cf, int col0)
+{
+    if constexpr (C != 0 && !WIDE) return RowGeom{C, C, 0};          // rows of exactly C channels
+    else if constexpr (C != 0) return RowGeom{C, cf, col0};           // blocks of C channels of wider rows
+    else return RowGeom{cw, cf, col0};
+}
 
 // Both elements of a packed bf16 pair: 2^23 + code as raw float bits (see biased_code()).  With
 // MASKED the value of a channel whose group is stored flat is replaced by 0 first, so that its
@@ -99,13 +116,14 @@ __device__ __forceinline__ void enc_release(uint64_t *empty_bar)
 // ---- level 0: the tile's rows as they are ------------------------------------------------------
 
 template <int C>
-__device__ __forceinline__ void enc_consume_raw(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
-                                             int nt, int tile, uint8_t *codes_sec)
+__device__ __forceinline__ void enc_consume_raw(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
+                                                int nt, int tile, uint8_t *codes_sec)
 {
-    const int c = C ? C : c_rt;
-    const int nvec = nt * (c >> 3);
+    const int vpr = g.cw >> 3;                            // 16-byte vectors per stage row
+    const int nvec = nt * vpr;
     const uint4 *src = reinterpret_cast<const uint4 *>(st);
-    uint4 *dst = reinterpret_cast<uint4 *>(codes_sec + 2 * (size_t)tile * kTileTokens * c);
+    uint8_t *dst = codes_sec + 2 * ((size_t)tile * kTileTokens * g.cf + g.col0);
+    const bool packed = g.cw == g.cf;                     // the tile's rows are contiguous in the stream too
     constexpr int U = 8;
     const int iters = (nvec + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);     // the same for every thread
     for (int it = 0; it < iters; ++it) {
@@ -116,8 +134,17 @@ __device__ __forceinline__ void enc_consume_raw(const uint8_t *st, int c_rt, int
             if (v0 + k * kEncGroupThreads < nvec) x[k] = src[v0 + k * kEncGroupThreads];
         if (it == iters - 1) enc_release(empty_bar);
 #pragma unroll
-        for (int k = 0; k < U; ++k)
-            if (v0 + k * kEncGroupThreads < nvec) __stcs(dst + v0 + k * kEncGroupThreads, x[k]);
+        for (int k = 0; k < U; ++k) {
+            const int v = v0 + k * kEncGroupThreads;
+            if (v < nvec) {
+                size_t off = 16 * (size_t)v;
+                if (!packed) {
+                    const int row = v / vpr;
+                    off = 2 * (size_t)row * g.cf + 16 * (size_t)(v - row * vpr);
+                }
+                __stcs(reinterpret_cast<uint4 *>(dst + off), x[k]);
+            }
+        }
     }
 }
 
@@ -156,23 +183,36 @@ __device__ __forceinline__ bool enc_params_k(uint32_t mn01, uint32_t mn23, uint3
     return all_quantised;
 }
 
+// Where the metadata words and the first row's codes of 4-channel column cq of a tile go.
+template <int BITS>
+__device__ __forceinline__ void enc_k_out(RowGeom g, int cq, int tile, uint8_t *meta_sec, uint8_t *codes_sec,
+                                          uint4 *&meta_out, uint8_t *&codes_out, uint32_t &row_bytes)
+{
+    const size_t ch = (size_t)g.col0 + 4 * (size_t)cq;   // the column's first channel within the plane
+    meta_out = reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * g.cf + ch));
+    codes_out = codes_sec + ((size_t)tile * kTileTokens * g.cf + ch) * BITS / 8;
+    row_bytes = (uint32_t)g.cf * BITS / 8;
+}
+
 // A full tile of K once its 32 rows of the thread's 4 channels (column cq) sit in registers:
 // ranges, metadata, codes.
-template <int BITS, int C>
-__device__ __forceinline__ void enc_process_k(uint2 (&x)[kTileTokens], int c_rt, int cq, int tile,
+template <int BITS>
+__device__ __forceinline__ void enc_process_k(uint2 (&x)[kTileTokens], RowGeom g, int cq, int tile,
                                               uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int c = C ? C : c_rt;
     uint32_t mn01 = x[0].x, mn23 = x[0].y, mx01 = x[0].x, mx23 = x[0].y;
 #pragma unroll
     for (int t = 1; t < kTileTokens; ++t) {
         mn01 = bmin2(mn01, x[t].x); mx01 = bmax2(mx01, x[t].x);
         mn23 = bmin2(mn23, x[t].y); mx23 = bmax2(mx23, x[t].y);
     }
+    uint4 *meta_out;
+    uint8_t *out;
+    uint32_t row_bytes;
+    enc_k_out<BITS>(g, cq, tile, meta_sec, codes_sec, meta_out, out, row_bytes);
     float lo[4], inv[4];
     uint32_t mask[4];
-    const bool all_quantised = enc_params_k<BITS>(
-        mn01, mn23, mx01, mx23, reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
+    const bool all_quantised = enc_params_k<BITS>(mn01, mn23, mx01, mx23, meta_out, lo, inv, mask);
     if (!all_quantised) {
         // a channel stored flat: its values become 0 so that (0 - min) * 0 is a zero and the code 0
         // (x - min may overflow for such a group, and infinity * 0 would be NaN)
@@ -183,20 +223,17 @@ __device__ __forceinline__ void enc_process_k(uint2 (&x)[kTileTokens], int c_rt,
     }
     const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
     const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
-    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-    uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
 #pragma unroll
     for (int t = 0; t < kTileTokens; ++t)
         enc_store_row_k<BITS, false>(x[t], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
 }
 
 // A full tile: all 32 rows of the thread's 4 channels in registers, one pass over shared memory.
-template <int BITS, int C>
-__device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+template <int BITS>
+__device__ __forceinline__ void enc_consume_k(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
                                               int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int c = C ? C : c_rt;
-    const int C4 = c >> 2;                               // 4-channel columns per row, <= 256
+    const int C4 = g.cw >> 2;                            // 4-channel columns per stage row, <= 256
     const bool active = tid < C4;
     const int cq = active ? tid : 0;
     const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
@@ -204,13 +241,13 @@ __device__ __forceinline__ void enc_consume_k(const uint8_t *st, int c_rt, int t
 #pragma unroll
     for (int t = 0; t < kTileTokens; ++t) x[t] = col[t * C4];
     enc_release(empty_bar);
-    if (active) enc_process_k<BITS, C>(x, c_rt, cq, tile, meta_sec, codes_sec);
+    if (active) enc_process_k<BITS>(x, g, cq, tile, meta_sec, codes_sec);
 }
 
 // The last, short tile of a chunk (nt < 32 rows): rare, so two plain passes over the rows.
 // row(t) returns row t of the thread's 4 channels (column cq) as two packed bf16 pairs.
 template <int BITS, typename RowFn>
-__device__ __forceinline__ void enc_k_short(RowFn row, int c, int cq, int nt, int tile,
+__device__ __forceinline__ void enc_k_short(RowFn row, RowGeom g, int cq, int nt, int tile,
                                             uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const uint2 x0 = row(0);
@@ -221,27 +258,28 @@ __device__ __forceinline__ void enc_k_short(RowFn row, int c, int cq, int nt, in
         mn01 = bmin2(mn01, x.x); mx01 = bmax2(mx01, x.x);
         mn23 = bmin2(mn23, x.y); mx23 = bmax2(mx23, x.y);
     }
+    uint4 *meta_out;
+    uint8_t *out;
+    uint32_t row_bytes;
+    enc_k_out<BITS>(g, cq, tile, meta_sec, codes_sec, meta_out, out, row_bytes);
     float lo[4], inv[4];
     uint32_t mask[4];
-    (void)enc_params_k<BITS>(mn01, mn23, mx01, mx23,
-                             reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)), lo, inv, mask);
+    (void)enc_params_k<BITS>(mn01, mn23, mx01, mx23, meta_out, lo, inv, mask);
     const f32x2 lo_a = f2_make(lo[0], lo[1]), lo_b = f2_make(lo[2], lo[3]);
     const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
-    const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-    uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BITS / 8;
 #pragma unroll 1
     for (int t = 0; t < nt; ++t)
         enc_store_row_k<BITS, true>(row(t), lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
 }
 
 template <int BITS>
-__device__ __noinline__ void enc_consume_k_short(const uint8_t *st, int c, int tid, uint64_t *empty_bar,
+__device__ __noinline__ void enc_consume_k_short(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
                                                  int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int C4 = c >> 2;
+    const int C4 = g.cw >> 2;
     if (tid < C4) {
         const uint2 *col = reinterpret_cast<const uint2 *>(st) + tid;
-        enc_k_short<BITS>([&](int t) { return col[t * C4]; }, c, tid, nt, tile, meta_sec, codes_sec);
+        enc_k_short<BITS>([&](int t) { return col[t * C4]; }, g, tid, nt, tile, meta_sec, codes_sec);
     }
     enc_release(empty_bar);
 }
@@ -324,20 +362,25 @@ __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32
                                                            __byte_perm(p[2][0], p[3][0], 0x5410));
 }
 
-template <int BITS, int C>
-__device__ __forceinline__ void enc_consume_v(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
-                                           int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+// Index, within the plane's V sections, of group gs of the tile's stage (stage rows hold cw / 32
+// groups, plane rows cf / 32).
+__device__ __forceinline__ size_t enc_v_group_index(RowGeom g, int tile, int gs)
 {
-    const int c = C ? C : c_rt;
-    const int gpr = c >> 5;                              // groups per row
-    const int ngroups = nt * gpr;                        // the tile's groups, in stream order
+    const int gpr_w = g.cw >> 5, gpr_f = g.cf >> 5;
+    const int row = gs / gpr_w;                          // a shift when the width is compiled in
+    return ((size_t)tile * kTileTokens + row) * gpr_f + (g.col0 >> 5) + (gs - row * gpr_w);
+}
+
+template <int BITS>
+__device__ __forceinline__ void enc_consume_v(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
+                                              int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+{
+    const int ngroups = nt * (g.cw >> 5);                // the tile's groups, in stage order
     const int rot = (tid >> 1) & 3;
     uint32_t off[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) off[j] = (uint32_t)((j + rot) & 3) * 16u;
-    const size_t g_first = (size_t)tile * kTileTokens * gpr;      // the tile's first group within the plane
-    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec) + g_first;
-    uint8_t *codes = codes_sec + g_first * (4 * BITS);
+    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec);
     constexpr int U = 2;                                 // groups a thread holds at a time
     const int iters = (ngroups + kEncGroupThreads * U - 1) / (kEncGroupThreads * U);  // the same for every thread
     for (int it = 0; it < iters; ++it) {
@@ -345,56 +388,60 @@ __device__ __forceinline__ void enc_consume_v(const uint8_t *st, int c_rt, int t
         uint4 x[U][4];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const int g = g0 + k * kEncGroupThreads;
-            if (g < ngroups) {
+            const int gs = g0 + k * kEncGroupThreads;
+            if (gs < ngroups) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) x[k][j] = *reinterpret_cast<const uint4 *>(st + (size_t)g * 64 + off[j]);
+                for (int j = 0; j < 4; ++j) x[k][j] = *reinterpret_cast<const uint4 *>(st + (size_t)gs * 64 + off[j]);
             }
         }
         if (it == iters - 1) enc_release(empty_bar);
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const int g = g0 + k * kEncGroupThreads;
-            if (g < ngroups) enc_group_v<BITS>(x[k], rot, enc_range_v(x[k]), meta + g, codes + (size_t)g * (4 * BITS));
+            const int gs = g0 + k * kEncGroupThreads;
+            if (gs < ngroups) {
+                const size_t gi = enc_v_group_index(g, tile, gs);
+                enc_group_v<BITS>(x[k], rot, enc_range_v(x[k]), meta + gi, codes_sec + gi * (4 * BITS));
+            }
         }
     }
 }
 
 // One unit of a known level: K or V (or the raw copy), inlined into the caller.
-template <int C, int LEVEL>
+template <int C, int LEVEL, bool WIDE = false>
 __device__ __forceinline__ void enc_consume_level(const EncUnit &u, const uint8_t *st, int c_rt, int tid,
                                                   uint64_t *eb)
 {
+    const RowGeom g = row_geom<C, WIDE>(u.cw, c_rt, u.col0);
     if constexpr (LEVEL == 0) {
-        enc_consume_raw<C>(st, c_rt, tid, eb, u.nt, u.tile, u.codes);
+        enc_consume_raw<C>(st, g, tid, eb, u.nt, u.tile, u.codes);
     } else {
         constexpr int BITS = 16 >> LEVEL;
-        if (u.kv) enc_consume_v<BITS, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
-        else if (u.nt == kTileTokens) enc_consume_k<BITS, C>(st, c_rt, tid, eb, u.tile, u.meta, u.codes);
-        else enc_consume_k_short<BITS>(st, C ? C : c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        if (u.kv) enc_consume_v<BITS>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        else if (u.nt == kTileTokens) enc_consume_k<BITS>(st, g, tid, eb, u.tile, u.meta, u.codes);
+        else enc_consume_k_short<BITS>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
     }
 }
 // The same as a function of its own: a kernel that has to hold all four levels keeps each level's
 // registers apart this way (inlined side by side they spill).
-template <int C, int LEVEL>
+template <int C, int LEVEL, bool WIDE>
 __device__ __noinline__ void enc_consume_level_call(const EncUnit *u, const uint8_t *st, int c_rt, int tid,
                                                     uint64_t *eb)
 {
-    enc_consume_level<C, LEVEL>(*u, st, c_rt, tid, eb);
+    enc_consume_level<C, LEVEL, WIDE>(*u, st, c_rt, tid, eb);
 }
 
 // LEVEL >= 0: every chunk of the launch has this level (checked by the producer); -1: any mix.
-template <int C, int LEVEL>
+template <int C, int LEVEL, bool WIDE>
 __device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st, int c_rt, int tid, uint64_t *eb)
 {
     if constexpr (LEVEL >= 0) {
-        enc_consume_level<C, LEVEL>(u, st, c_rt, tid, eb);
+        enc_consume_level<C, LEVEL, WIDE>(u, st, c_rt, tid, eb);
     } else {
         switch (u.bits) {                                // uniform per consumer group
-        case 16: enc_consume_level_call<C, 0>(&u, st, c_rt, tid, eb); break;
-        case 8: enc_consume_level_call<C, 1>(&u, st, c_rt, tid, eb); break;
-        case 4: enc_consume_level_call<C, 2>(&u, st, c_rt, tid, eb); break;
-        default: enc_consume_level_call<C, 3>(&u, st, c_rt, tid, eb); break;
+        case 16: enc_consume_level_call<C, 0, WIDE>(&u, st, c_rt, tid, eb); break;
+        case 8: enc_consume_level_call<C, 1, WIDE>(&u, st, c_rt, tid, eb); break;
+        case 4: enc_consume_level_call<C, 2, WIDE>(&u, st, c_rt, tid, eb); break;
+        default: enc_consume_level_call<C, 3, WIDE>(&u, st, c_rt, tid, eb); break;
         }
     }
 }
@@ -403,7 +450,7 @@ __device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st
 //        1 = one CTA per tile in the grid, running CTAs pull further tiles through cluster launch control.
 // The 8 consumer warps take every unit together: a stage's full barrier is then waited on once per
 // phase, which is what lets one parity bit tell the phases apart.
-template <int C, int LEVEL, typename Chunks>
+template <int C, int LEVEL, typename Chunks, bool WIDE = false>
 __global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
 encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, const Chunks chunks)
 {
@@ -432,7 +479,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
 
     if (warp == kProducerWarp) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
         uint32_t unit = 0;
         bool ok = true;
 
@@ -445,8 +492,10 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int tile = (int)(tile_id % kTilesPerChunk);
-            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share rows
+            const int64_t row_tile = tile_id / p.n_blocks;
+            const int tile = (int)(row_tile % kTilesPerChunk);
+            const int64_t plane_id = row_tile / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), p.chunk0);
@@ -476,31 +525,45 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
             const int64_t j0 = tok0 + tile * kTileTokens;        // the tile's first token in the encoded sequence
             ok = acquire();
             if (!ok) return;
+            const int s = unit % kEncStages;
+            uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+            const uint32_t row_bytes = 2u * (uint32_t)p.bw;                     // a multiple of 64
             if (lane == 0) {
-                const int s = unit % kEncStages;
                 EncUnit &u = info[s];
                 u.bits = level_bits(d.level); u.kv = kv; u.nt = nt; u.tile = tile;
-                u.last = tile * kTileTokens + nt == n;
+                u.last = tile * kTileTokens + nt == n && cb == p.n_blocks - 1;
                 u.meta_payload = (uint32_t)(kv ? L.vmeta_payload : L.kmeta_payload);
                 u.meta_padded = (uint32_t)(kv ? L.vmeta : L.kmeta);
                 u.codes_payload = (uint32_t)L.codes_payload;
                 u.codes_padded = (uint32_t)L.kcodes;
                 u.meta = lay + L.meta_off(kv);
                 u.codes = lay + L.codes_off(kv);
-                const uint32_t row_bytes = 2u * (uint32_t)p.c;                  // a multiple of 64
-                uint8_t *st = stage_mem + (size_t)s * kEncStageBytes;
+                u.col0 = cb * p.bw; u.cw = p.bw;
                 mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nt * row_bytes);
-                if (p.n_runs == 0) {
-                    bulk_load(st, plane + j0 * p.c, (uint32_t)nt * row_bytes, &full_bar[s]);
-                } else {
-                    // token dropping: the tile's rows come from the kept runs it overlaps, one copy per run
-                    for (int r = 0; r < p.n_runs; ++r) {
-                        const int64_t a = max(j0, p.run_pos[r]), b = min(j0 + nt, p.run_pos[r + 1]);
-                        if (a < b)
-                            bulk_load(st + (size_t)(a - j0) * row_bytes,
-                                      plane + (p.run_first[r] + (a - p.run_pos[r])) * p.c,
-                                      (uint32_t)(b - a) * row_bytes, &full_bar[s]);
+            }
+            if (p.n_blocks == 1) {
+                if (lane == 0) {
+                    if (p.n_runs == 0) {
+                        bulk_load(st, plane + j0 * p.c, (uint32_t)nt * row_bytes, &full_bar[s]);
+                    } else {
+                        // token dropping: the tile's rows come from the kept runs it overlaps, one copy per run
+                        for (int r = 0; r < p.n_runs; ++r) {
+                            const int64_t a = max(j0, p.run_pos[r]), b = min(j0 + nt, p.run_pos[r + 1]);
+                            if (a < b)
+                                bulk_load(st + (size_t)(a - j0) * row_bytes,
+                                          plane + (p.run_first[r] + (a - p.run_pos[r])) * p.c,
+                                          (uint32_t)(b - a) * row_bytes, &full_bar[s]);
+                        }
                     }
+                }
+            } else {
+                // a column block of wide rows: lane r copies row r's piece (the expectation is posted first)
+                __syncwarp();
+                if (lane < nt) {
+                    int64_t tok = j0 + lane;                                    // in the encoded sequence
+                    for (int r = 0; r < p.n_runs; ++r)
+                        if (tok >= p.run_pos[r] && tok < p.run_pos[r + 1]) { tok = p.run_first[r] + (tok - p.run_pos[r]); break; }
+                    bulk_load(st + (size_t)lane * row_bytes, plane + tok * p.c + cb * p.bw, row_bytes, &full_bar[s]);
                 }
             }
             ++unit;
@@ -576,7 +639,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                 if (u.codes_payload + tid < u.codes_padded) u.codes[u.codes_payload + tid] = 0;
                 if (u.bits < 16 && u.meta_payload + tid < u.meta_padded) u.meta[u.meta_payload + tid] = 0;
             }
-            enc_dispatch<C, LEVEL>(u, st, p.c, tid, eb);
+            enc_dispatch<C, LEVEL, WIDE>(u, st, p.c, tid, eb);
         }
     }
 }

@@ -38,6 +38,17 @@ inline unsigned grid_for(int64_t n_chunks, int l)
     return (g <= 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;
 }
 
+// Width of the column blocks the TMA-fed kernels cut a row of c channels into: c itself up to 1024,
+// else the largest divisor of c that is at most 1024 and a multiple of 128 (every piece a bulk copy
+// moves is then a multiple of 16 bytes), or 0 if there is none.
+inline int block_width(int c)
+{
+    if (c <= 1024) return c;
+    for (int w = 1024; w >= 128; w -= 128)
+        if (c % w == 0) return w;
+    return 0;
+}
+
 inline kvh_status launch_status()
 {
     return cudaPeekAtLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;

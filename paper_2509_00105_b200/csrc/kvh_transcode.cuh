@@ -304,6 +304,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
                 u.e.codes_padded = (uint32_t)Lo.kcodes;
                 u.e.meta = lay_out + Lo.meta_off(kv);
                 u.e.codes = lay_out + Lo.codes_off(kv);
+                u.e.col0 = 0; u.e.cw = p.c;
                 uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
                 const uint8_t *codes_in = lay_in + Li.codes_off(kv);
                 if (di.level == 0) {

@@ -83,6 +83,7 @@ SHAPES = [
     # l, c, N
     (1, 32, 1), (1, 32, 15), (2, 32, 16), (1, 64, 17), (1, 96, 31), (1, 128, 32), (2, 160, 33),
     (1, 256, 255), (1, 32, 256), (2, 64, 257), (1, 1024, 300), (1, 2048, 40), (1, 4096, 33), (3, 512, 700),
+    (1, 1152, 70), (1, 1280, 33), (2, 3072, 290), (1, 2080, 35),     # wider than 1024: column blocks of 384, 640, 1024; none
 ]
 
 

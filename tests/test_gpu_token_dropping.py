@@ -20,6 +20,9 @@ CASES = [
     (2, 512, 300, [(0, 300)], 1),                        # nothing dropped
     (1, 1024, 5000, [(4999, 1)], 3),                     # a single kept token
     (1, 64, 600, [(0, 33), (567, 33)], 0),               # level 0: kept rows as they are
+    (1, 2048, 300, [(0, 4), (100, 60)], 2),              # rows wider than a stage: column blocks of 1024
+    (1, 1152, 200, [(3, 30), (150, 41)], [1]),           # ... of 384
+    (1, 3072, 90, [(0, 90)], 0),
 ]
 
 
@@ -108,8 +111,8 @@ def test_encode_kept_rejects_bad_runs(kvh):
     with pytest.raises(kvh.KvhError) as e:
         kvh.encode_kept(kv, R([(0, 100)]), None, len(descs), out[:total - 128], level=1)
     assert e.value.status == 5
-    wide = workloads.make_kv(1, 40, 2048, seed=2, device="cuda")
-    d2, t2 = kvh.plan_chunks(1, 2048, 8, 1)
+    wide = workloads.make_kv(1, 40, 2080, seed=2, device="cuda")      # 65 x 32 channels: no column-block width fits
+    d2, t2 = kvh.plan_chunks(1, 2080, 8, 1)
     with pytest.raises(kvh.KvhError) as e:
         kvh.encode_kept(wide, R([(0, 8)]), kvh.descs_to_tensor(d2, "cuda"), 1, torch.empty(t2, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 3
