@@ -173,7 +173,7 @@ def test_launches_too_large_for_a_grid_and_new_entry_points_reject_before_any_cu
     assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 1, -1, a, 1 << 20, None, None) == 1   # no descriptors, no level
     assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 2, 1, a, 1 << 20, None, None) == 3    # 10 kept tokens = 1 chunk
     assert L.kvh_encode_kept(a, 1, 100, 32, runs, 1, None, 1, 1, a, 64, None, None) == 5
-    assert L.kvh_encode_kept(a, 1, 100, 2048, runs, 1, None, 1, 1, a, 1 << 20, None, None) == 3
+    assert L.kvh_encode_kept(a, 1, 100, 2080, runs, 1, None, 1, 1, a, 1 << 20, None, None) == 3      # 65 x 32: no block width
     # policy: arguments
     assert L.kvh_policy_assign(None, a, a, 1, a, a, None, None) == 1
     tier = np.array([(1.0, 0.0, 100)], dtype=kvh.TIER_DTYPE)                      # bandwidth must be positive
