@@ -37,12 +37,15 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     // persistent TMA kernel needs a tile to fit a shared-memory stage and at most 2 pages per tile.
     const char *force = getenv("KVH_DECODE_PATH");
     const bool want_tma = !(force && strcmp(force, "direct") == 0);
-    if (want_tma && p.c <= kTmaMaxChannels && p.page_tokens >= 16) {
+    p.bw = block_width(p.c);                             // rows wider than 1024 channels go in column blocks
+    p.n_blocks = p.bw > 0 ? p.c / p.bw : 1;
+    const int64_t tiles = (int64_t)grid * p.n_blocks;
+    if (want_tma && p.bw > 0 && tiles <= 0x7fffffffLL && p.page_tokens >= 16) {
         int dev = 0, sms = 0, per_sm = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return KVH_ERR_CUDA;
-        const uint32_t stage = tma_stage_bytes(p.c);
+        const uint32_t stage = tma_stage_bytes(p.bw);
         int stages = (int)((112u * 1024u) / stage);           // two CTAs per SM when c = 1024
         stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
         const size_t dyn = (size_t)stages * stage;
@@ -57,7 +60,7 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         const char *sched_env = getenv("KVH_DECODE_SCHED");
         const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
         const int64_t resident = (int64_t)sms * per_sm;
-        const unsigned pgrid = sched == 1 ? grid : (unsigned)(grid < resident ? grid : resident);
+        const unsigned pgrid = sched == 1 ? (unsigned)tiles : (unsigned)(tiles < resident ? tiles : resident);
         kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
         return launch_status();
     }

@@ -26,6 +26,7 @@ struct DecodeParams {
     uint16_t *pool;
     int64_t layer_stride, kv_stride, page_stride;
     int32_t num_pages, page_tokens, page_shift, l, c;   // page_tokens == 1 << page_shift
+    int32_t bw, n_blocks;             // TMA-fed kernel: channels per column block (c when c <= 1024), blocks per row
     int32_t *status;
 };
 

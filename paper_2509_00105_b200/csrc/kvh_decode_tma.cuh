@@ -33,6 +33,7 @@ struct UnitInfo {
     int32_t nrows;       // tokens in the unit (1..32)
     int32_t pg0, pg1;    // page ids of the page holding row0 and of the next one
     uint16_t *plane;     // pool + layer*layer_stride + kv*kv_stride
+    int32_t col0, cw;    // first channel and width of the unit's column block (0, c unless rows exceed 1024 channels)
 };
 
 __host__ __device__ __forceinline__ uint32_t tma_stage_bytes(int c) { return (36u * (uint32_t)c + 127u) & ~127u; }
@@ -120,7 +121,7 @@ struct RowRun {
 template <int C>
 __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u)
 {
-    const int V8 = (C ? C : p.c) >> 3;                              // <= 128
+    const int V8 = (C ? C : u.cw) >> 3;                   // 16-byte vectors per stage row, <= 128
     const int rpp = kConsumerThreads / V8;                // row groups the CTA holds, >= 2
     int rpt = 1;
     while (rpt * rpp < kTileTokens) rpt <<= 1;            // rows per thread: 16 when c = 1024
@@ -134,7 +135,7 @@ __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo 
         const int T = u.row0 + r.first;
         const int32_t pg = (T >> p.page_shift) == (u.row0 >> p.page_shift) ? u.pg0 : u.pg1;
         r.dst = page_row<C>(p, pg, u.plane, T);              // reports an out-of-range page id
-        if (r.dst) r.dst += 8 * r.cv; else r.count = 0;
+        if (r.dst) r.dst += (C ? 0 : u.col0) + 8 * r.cv; else r.count = 0;
     }
     return r;
 }
@@ -142,20 +143,21 @@ __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo 
 template <int C>
 __device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
 {
-    const int c = C ? C : p.c;
+    const int cw = C ? C : u.cw;                          // row width in the stage
     const RowRun r = row_run<C>(p, u);
-    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * c + 8 * r.cv));
+    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * cw + 8 * r.cv));
     uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
-    const int stride = c >> 3;                            // uint4 per row
+    const int sstride = cw >> 3, dstride = (C ? C : p.c) >> 3;    // uint4 per stage row / per page row
 #pragma unroll 4
-    for (int k = 0; k < r.count; ++k) dst[(size_t)k * stride] = src[(size_t)k * stride];
+    for (int k = 0; k < r.count; ++k) dst[(size_t)k * dstride] = src[(size_t)k * sstride];
 }
 
 template <int BITS, int C>
 __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
-    const int c = C ? C : p.c;
+    const int c = C ? C : u.cw;                           // row width in the stage
+    const int dstride = C ? C : p.c;                      // row width of a page
     const RowRun r = row_run<C>(p, u);
     if (r.count == 0) return;
     f32x2 lo[4], sc[4];
@@ -184,7 +186,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
         spread8<BITS>(src, x);
         *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
         src += row_bytes;
-        dst += c;
+        dst += dstride;
     }
 }
 
@@ -192,7 +194,8 @@ template <int BITS, int C>
 __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
-    const int c = C ? C : p.c;
+    const int c = C ? C : u.cw;                           // row width in the stage
+    const int dstride = C ? C : p.c;                      // row width of a page
     const RowRun r = row_run<C>(p, u);
     const int lane = threadIdx.x & 31;
     const uint32_t quad = 0xfu << (lane & ~3);            // the 4 lanes that share every V group
@@ -224,7 +227,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
                 spread8<BITS>(src, x);
                 *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
                 src += row_bytes;
-                dst += c;
+                dst += dstride;
             }
         }
     }
@@ -245,8 +248,8 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
 
-    const uint32_t stage_bytes = tma_stage_bytes(p.c);
-    const uint32_t meta_off = 32u * p.c;
+    const uint32_t stage_bytes = tma_stage_bytes(p.bw);
+    const uint32_t meta_off = 32u * p.bw;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -263,7 +266,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
 
     if (warp == kConsumerThreads / 32) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
         int cur_chunk = -1;
         bool valid = false;
         kvh_chunk_desc d = p.single;
@@ -272,8 +275,13 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
         uint32_t unit = 0;
         bool ok = true;
 
-        auto emit = [&](int bits, int kv, int row0, int nrows, uint16_t *plane, const uint8_t *codes_src,
-                        uint32_t codes_bytes, const uint8_t *meta_src, uint32_t meta_bytes) -> bool {
+        // One unit.  Contiguous source (rows as wide as the plane): one copy of codes_bytes and one of
+        // meta_bytes.  A column block of wider rows (row_stride != 0): lane r copies row r's codes_bytes
+        // from codes_src + r * row_stride and, for V, its meta_bytes from meta_src + r * mrow_stride
+        // (K metadata is one piece: mrow_stride == 0).
+        auto emit = [&](int bits, int kv, int row0, int nrows, uint16_t *plane, int col0, const uint8_t *codes_src,
+                        uint32_t codes_bytes, uint32_t row_stride, const uint8_t *meta_src, uint32_t meta_bytes,
+                        uint32_t mrow_stride) -> bool {
             const int s = unit % n_stages;
             if (unit >= (uint32_t)n_stages) {
                 bool w = true;
@@ -284,16 +292,32 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const int pidx = row0 >> p.page_shift;
             const int32_t pg0 = __shfl_sync(0xffffffffu, my_pg, pidx & 31);
             const int32_t pg1 = __shfl_sync(0xffffffffu, my_pg, (pidx + 1) & 31);
+            uint8_t *st = stage_mem + (size_t)s * stage_bytes;
+            const bool strided = row_stride != 0;
             if (lane == 0) {
                 UnitInfo &u = info[s];
                 u.bits = bits; u.kv = kv; u.row0 = row0; u.nrows = nrows; u.pg0 = pg0; u.pg1 = pg1; u.plane = plane;
-                uint8_t *st = stage_mem + (size_t)s * stage_bytes;
+                u.col0 = col0; u.cw = p.bw;
                 if (bits == 0) {
                     mbar_arrive(&full_bar[s]);
-                } else {
+                } else if (!strided) {
                     mbar_arrive_expect_tx(&full_bar[s], codes_bytes + meta_bytes);
                     bulk_load(st, codes_src, codes_bytes, &full_bar[s]);
                     if (meta_bytes) bulk_load(st + meta_off, meta_src, meta_bytes, &full_bar[s]);
+                } else {
+                    const uint32_t meta_total = mrow_stride ? (uint32_t)nrows * meta_bytes : meta_bytes;
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nrows * codes_bytes + meta_total);
+                    if (meta_bytes && !mrow_stride) bulk_load(st + meta_off, meta_src, meta_bytes, &full_bar[s]);
+                }
+            }
+            if (strided && bits != 0) {
+                __syncwarp();                            // the expectation is posted before any piece lands
+                if (lane < nrows) {
+                    bulk_load(st + (size_t)lane * codes_bytes, codes_src + (size_t)lane * row_stride, codes_bytes,
+                              &full_bar[s]);
+                    if (meta_bytes && mrow_stride)
+                        bulk_load(st + meta_off + (size_t)lane * meta_bytes, meta_src + (size_t)lane * mrow_stride,
+                                  meta_bytes, &full_bar[s]);
                 }
             }
             ++unit;
@@ -301,8 +325,10 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int tile = (int)(tile_id % kTilesPerChunk);
-            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share page rows
+            const int64_t row_tile = tile_id / p.n_blocks;
+            const int tile = (int)(row_tile % kTilesPerChunk);
+            const int64_t plane_id = row_tile / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = (int)((plane_id >> 1) / p.l);
@@ -329,19 +355,31 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const uint8_t *meta = lay + L.meta_off(kv);
             const uint8_t *codes = lay + L.codes_off(kv);
             uint16_t *plane = p.pool + (int64_t)layer * p.layer_stride + (int64_t)kv * p.kv_stride;
+            const bool wide = p.n_blocks > 1;
+            const int col0 = cb * p.bw;
+            const uint32_t gpr = (uint32_t)p.c / kGroup;         // groups per plane row
             if (d.level == 0) {
                 for (int h = 0; ok && h < nt; h += 16) {
                     const int rows = min(16, nt - h);
-                    ok = emit(16, kv, t0 + h, rows, plane, codes + 2 * (uint64_t)(t0 + h) * p.c,
-                              round16(2u * rows * p.c), nullptr, 0);
+                    const uint8_t *src = codes + 2 * ((uint64_t)(t0 + h) * p.c + col0);
+                    ok = wide ? emit(16, kv, t0 + h, rows, plane, col0, src, 2u * p.bw, 2u * p.c, nullptr, 0, 0)
+                              : emit(16, kv, t0 + h, rows, plane, 0, src, round16(2u * rows * p.c), 0, nullptr, 0, 0);
                 }
             } else {
                 const int b = level_bits(d.level);
-                const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
-                const uint8_t *msrc = kv == 0 ? meta + 4 * (uint64_t)tile * p.c
-                                              : meta + 4 * (uint64_t)t0 * (p.c / kGroup);
-                const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * (p.c / kGroup));
-                ok = emit(b, kv, t0, nt, plane, codes + (uint64_t)t0 * p.c * b / 8, cbytes, msrc, mbytes);
+                const uint8_t *csrc = codes + ((uint64_t)t0 * p.c + col0) * b / 8;
+                const uint8_t *msrc = kv == 0 ? meta + 4 * ((uint64_t)tile * p.c + col0)
+                                              : meta + 4 * ((uint64_t)t0 * gpr + col0 / kGroup);
+                if (wide) {
+                    ok = kv == 0 ? emit(b, kv, t0, nt, plane, col0, csrc, (uint32_t)p.bw * b / 8, (uint32_t)p.c * b / 8,
+                                        msrc, 4u * p.bw, 0)
+                                 : emit(b, kv, t0, nt, plane, col0, csrc, (uint32_t)p.bw * b / 8, (uint32_t)p.c * b / 8,
+                                        msrc, 4u * (p.bw / kGroup), 4u * gpr);
+                } else {
+                    const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
+                    const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * gpr);
+                    ok = emit(b, kv, t0, nt, plane, 0, csrc, cbytes, 0, msrc, mbytes, 0);
+                }
             }
         };
 
@@ -376,7 +414,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                 tile_id += gridDim.x;
             }
         }
-        if (ok) ok = emit(0, 0, 0, 0, nullptr, nullptr, 0, nullptr, 0);       // end marker
+        if (ok) ok = emit(0, 0, 0, 0, nullptr, 0, nullptr, 0, 0, nullptr, 0, 0);      // end marker
         if (!ok && lane == 0) {
             report(p.status, KVH_ERR_TIMEOUT);
             abort_flag = 1;

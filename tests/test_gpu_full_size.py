@@ -83,6 +83,12 @@ def test_llama8b_128k_offsets_beyond_32_bits(kvh):
     run_context(kvh, s, seed=5000, levels=(0, 3), sample=[0, 300, 511])
 
 
+def test_wide_rows_llama2_7b_shape(kvh):
+    """32 KV heads x 128 = 4096 channels: the TMA-fed kernels work in column blocks of 1024."""
+    s = workloads.LLAMA2_7B_4K
+    run_context(kvh, s, seed=7000, levels=(0, 1, 2, 3), sample=[0, 15])
+
+
 def test_batched_mixed_level_load_at_scale(kvh):
     """The batched mixed-level workload at its full size: 64 contexts of the 8B shape (32 layers),
     lengths log-uniform in [2K, 32K] with partial last chunks, a random level per chunk, one shared

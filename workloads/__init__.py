@@ -33,6 +33,8 @@ TINY = Shape("tiny", 4, 1024, 256)
 LLAMA8B_8K = Shape("llama3-8b-8k", 32, 1024, 8192)
 LLAMA70B_32K = Shape("llama3-70b-32k", 80, 1024, 32768)
 LLAMA8B_128K = Shape("llama3-8b-128k", 32, 1024, 131072)
+# a multi-head model without grouped KV heads (32 heads x 128): rows wider than the 1024 of the Llama-3 shapes
+LLAMA2_7B_4K = Shape("llama2-7b-4k", 32, 4096, 4096)
 BATCH_N_CONTEXTS = 64
 BATCH_MIN_TOKENS = 2048
 BATCH_MAX_TOKENS = 32768
