@@ -1,6 +1,8 @@
 // Host side of the C ABI declared in include/kvh.h: argument validation, size
 // arithmetic and kernel launches.  No device memory is allocated here and no
 // state survives a call.
+#include <cuda.h>
+#include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -71,6 +73,29 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
 // Encode launch: the persistent TMA-fed kernel when a 32-token tile fits a shared-memory stage,
 // otherwise one CTA per tile reading global memory directly.  KVH_ENCODE_PATH=direct forces the
 // latter and KVH_ENCODE_SCHED=static a fixed tile stride (measurement aids).
+// Tensor map of the encode source seen as a 2-D tensor [n_layers * 2 * src_N rows][c channels] of
+// bf16, with boxes of 256 channels x 32 rows; false if the driver entry point is not to be had.
+bool make_kv_map(const EncodeParams &p, CUtensorMap *map)
+{
+    static PFN_cuTensorMapEncodeTiled encode = [] {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+    }();
+    if (!encode) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)p.c, (cuuint64_t)p.l * 2 * (cuuint64_t)p.src_N};
+    const cuuint64_t strides[1] = {(cuuint64_t)p.c * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBoxChannels, (cuuint32_t)kTileTokens};
+    const cuuint32_t elem[2] = {1, 1};
+    if (dims[1] > 0xffffffffull) return false;
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(p.kv), dims, strides, box, elem,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <typename Chunks>
 kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, int n_chunks, cudaStream_t st,
                              const Chunks &chunks)
@@ -80,12 +105,16 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return KVH_ERR_CUDA;
     const size_t dyn = (size_t)kEncStages * kEncStageBytes;
-    void (*kernel)(const EncodeParams, const int, const int, const Chunks);
+    void (*kernel)(const EncodeParams, const int, const int, const Chunks, const CUtensorMap);
+    CUtensorMap kv_map{};
+    // wider rows in blocks of 1024 channels: the instance with the boxed stage; it wants the tensor
+    // map unless tokens are gathered from kept runs
+    const bool boxed = p.c != 1024 && p.bw == 1024 && (p.n_runs > 0 || make_kv_map(p, &kv_map));
     if (p.c == 1024) {
         kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks> : level == 1 ? encode_tma_kernel<1024, 1, Chunks>
                : level == 2 ? encode_tma_kernel<1024, 2, Chunks> : level == 3 ? encode_tma_kernel<1024, 3, Chunks>
                : encode_tma_kernel<1024, -1, Chunks>;
-    } else if (p.bw == 1024) {                           // wider rows in blocks of 1024 channels
+    } else if (boxed) {
         kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks, true> : level == 1 ? encode_tma_kernel<1024, 1, Chunks, true>
                : level == 2 ? encode_tma_kernel<1024, 2, Chunks, true> : level == 3 ? encode_tma_kernel<1024, 3, Chunks, true>
                : encode_tma_kernel<1024, -1, Chunks, true>;
@@ -99,7 +128,7 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
     const char *sched_env = getenv("KVH_ENCODE_SCHED");
     const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
     const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
-    kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, n_chunks, sched, chunks);
+    kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, n_chunks, sched, chunks, kv_map);
     return launch_status();
 }
 

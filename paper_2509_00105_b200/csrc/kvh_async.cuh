@@ -59,6 +59,15 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
+// 2-D tiled TMA load: the box the tensor map describes, with its corner at element (x, y) of the
+// tensor, lands packed (row after row) at dst; its full size counts on the mbarrier, rows or columns
+// outside the tensor arrive as zeros.  x times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tensor_load_2d(void *dst, const void *tensor_map, int x, int y, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_addr(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
+}
+
 // Cluster launch control (sm_100): a running CTA asks the hardware for the index of a CTA of this
 // grid that has not started yet and takes over its work; the 16-byte answer arrives in shared
 // memory and completes 16 bytes of transaction on the mbarrier.  Dynamic scheduling of a persistent

@@ -23,6 +23,8 @@
 // waits for its copies in flight and leaves.
 #pragma once
 
+#include <cuda.h>      // CUtensorMap
+
 #include "kvh_async.cuh"
 #include "kvh_encode.cuh"
 #include "kvh_format.cuh"
@@ -63,15 +65,27 @@ struct EncUnit {
 // multiple of 128); a tile is then 32 tokens of one block.  In the stage its rows are cw channels
 // wide and packed; in the plane (source and stream) rows are cf channels wide and the block starts
 // at channel col0.  With the channel count compiled in, all three are constants.
+// Blocks of 1024 channels arrive through 2-D tiled TMA as 4 boxes of 256 channels x 32 rows
+// (a box dimension is at most 256 elements): the stage is then [box][row][256 channels] (boxed)
+// instead of [row][cw channels].
+constexpr int kBoxChannels = 256;
+constexpr uint32_t kBoxBytes = 2u * kBoxChannels * kTileTokens;      // 16 KiB
 struct RowGeom {
     int cw, cf, col0;
+    bool boxed;
+    // byte offset in the stage of channel ch (a multiple of 4) of row 0, and between rows
+    __device__ __forceinline__ uint32_t stage_col(int ch) const
+    {
+        return boxed ? (uint32_t)(ch / kBoxChannels) * kBoxBytes + 2u * (uint32_t)(ch % kBoxChannels) : 2u * (uint32_t)ch;
+    }
+    __device__ __forceinline__ uint32_t stage_row_bytes() const { return boxed ? 2u * kBoxChannels : 2u * (uint32_t)cw; }
 };
 template <int C, bool WIDE = false>
 __device__ __forceinline__ RowGeom row_geom(int cw, int cf, int col0)
 {
-    if constexpr (C != 0 && !WIDE) return RowGeom{C, C, 0};          // rows of exactly C channels
-    else if constexpr (C != 0) return RowGeom{C, cf, col0};           // blocks of C channels of wider rows
-    else return RowGeom{cw, cf, col0};
+    if constexpr (C != 0 && !WIDE) return RowGeom{C, C, 0, false};        // rows of exactly C channels
+    else if constexpr (C != 0) return RowGeom{C, cf, col0, true};         // blocks of C = 1024 channels of wider rows
+    else return RowGeom{cw, cf, col0, false};
 }
 
 // Both elements of a packed bf16 pair: 2^23 + code as raw float bits (see biased_code()).  With
@@ -130,8 +144,17 @@ __device__ __forceinline__ void enc_consume_raw(const uint8_t *st, RowGeom g, in
         const int v0 = it * kEncGroupThreads * U + tid;
         uint4 x[U];
 #pragma unroll
-        for (int k = 0; k < U; ++k)
-            if (v0 + k * kEncGroupThreads < nvec) x[k] = src[v0 + k * kEncGroupThreads];
+        for (int k = 0; k < U; ++k) {
+            const int v = v0 + k * kEncGroupThreads;
+            if (v < nvec) {
+                if (g.boxed) {
+                    const int row = v / vpr;
+                    x[k] = *reinterpret_cast<const uint4 *>(st + g.stage_col(8 * (v - row * vpr)) + row * g.stage_row_bytes());
+                } else {
+                    x[k] = src[v];
+                }
+            }
+        }
         if (it == iters - 1) enc_release(empty_bar);
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -236,10 +259,11 @@ __device__ __forceinline__ void enc_consume_k(const uint8_t *st, RowGeom g, int 
     const int C4 = g.cw >> 2;                            // 4-channel columns per stage row, <= 256
     const bool active = tid < C4;
     const int cq = active ? tid : 0;
-    const uint2 *col = reinterpret_cast<const uint2 *>(st) + cq;
+    const uint8_t *col = st + g.stage_col(4 * cq);
+    const uint32_t rs = g.stage_row_bytes();
     uint2 x[kTileTokens];
 #pragma unroll
-    for (int t = 0; t < kTileTokens; ++t) x[t] = col[t * C4];
+    for (int t = 0; t < kTileTokens; ++t) x[t] = *reinterpret_cast<const uint2 *>(col + t * rs);
     enc_release(empty_bar);
     if (active) enc_process_k<BITS>(x, g, cq, tile, meta_sec, codes_sec);
 }
@@ -278,8 +302,10 @@ __device__ __noinline__ void enc_consume_k_short(const uint8_t *st, RowGeom g, i
 {
     const int C4 = g.cw >> 2;
     if (tid < C4) {
-        const uint2 *col = reinterpret_cast<const uint2 *>(st) + tid;
-        enc_k_short<BITS>([&](int t) { return col[t * C4]; }, g, tid, nt, tile, meta_sec, codes_sec);
+        const uint8_t *col = st + g.stage_col(4 * tid);
+        const uint32_t rs = g.stage_row_bytes();
+        enc_k_short<BITS>([&](int t) { return *reinterpret_cast<const uint2 *>(col + t * rs); }, g, tid, nt, tile,
+                          meta_sec, codes_sec);
     }
     enc_release(empty_bar);
 }
@@ -375,7 +401,8 @@ template <int BITS>
 __device__ __forceinline__ void enc_consume_v(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
                                               int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int ngroups = nt * (g.cw >> 5);                // the tile's groups, in stage order
+    const int gpr_w = g.cw >> 5;
+    const int ngroups = nt * gpr_w;                      // the tile's groups, in stage order
     const int rot = (tid >> 1) & 3;
     uint32_t off[4];
 #pragma unroll
@@ -390,8 +417,11 @@ __device__ __forceinline__ void enc_consume_v(const uint8_t *st, RowGeom g, int 
         for (int k = 0; k < U; ++k) {
             const int gs = g0 + k * kEncGroupThreads;
             if (gs < ngroups) {
+                const int row = gs / gpr_w;              // boxed: 8 groups per box row
+                const uint8_t *grp = g.boxed ? st + g.stage_col(32 * (gs - row * gpr_w)) + row * g.stage_row_bytes()
+                                             : st + (size_t)gs * 64;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) x[k][j] = *reinterpret_cast<const uint4 *>(st + (size_t)gs * 64 + off[j]);
+                for (int j = 0; j < 4; ++j) x[k][j] = *reinterpret_cast<const uint4 *>(grp + off[j]);
             }
         }
         if (it == iters - 1) enc_release(empty_bar);
@@ -452,7 +482,8 @@ __device__ __forceinline__ void enc_dispatch(const EncUnit &u, const uint8_t *st
 // phase, which is what lets one parity bit tell the phases apart.
 template <int C, int LEVEL, typename Chunks, bool WIDE = false>
 __global__ void __launch_bounds__(32 + kEncGroupThreads, 1)
-encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, const Chunks chunks)
+encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, const Chunks chunks,
+                  const __grid_constant__ CUtensorMap kv_map)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kEncStages];
@@ -539,7 +570,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                 u.meta = lay + L.meta_off(kv);
                 u.codes = lay + L.codes_off(kv);
                 u.col0 = cb * p.bw; u.cw = p.bw;
-                mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nt * row_bytes);
+                mbar_arrive_expect_tx(&full_bar[s], WIDE && p.n_runs == 0 ? 4 * kBoxBytes : (uint32_t)nt * row_bytes);
             }
             if (p.n_blocks == 1) {
                 if (lane == 0) {
@@ -556,6 +587,16 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                         }
                     }
                 }
+            } else if (WIDE && p.n_runs == 0) {
+                // blocks of 1024 channels of wider rows: 4 boxes of 256 channels x 32 rows through the
+                // tensor map of the source seen as [planes * tokens][c]; rows past the tile are loaded too
+                // (zeros past the tensor's end) and ignored
+                if (lane == 0) {
+                    const int row = (int)(((int64_t)layer * 2 + kv) * p.src_N + j0);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        tensor_load_2d(st + k * kBoxBytes, &kv_map, cb * p.bw + k * kBoxChannels, row, &full_bar[s]);
+                }
             } else {
                 // a column block of wide rows: lane r copies row r's piece (the expectation is posted first)
                 __syncwarp();
@@ -563,7 +604,15 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                     int64_t tok = j0 + lane;                                    // in the encoded sequence
                     for (int r = 0; r < p.n_runs; ++r)
                         if (tok >= p.run_pos[r] && tok < p.run_pos[r + 1]) { tok = p.run_first[r] + (tok - p.run_pos[r]); break; }
-                    bulk_load(st + (size_t)lane * row_bytes, plane + tok * p.c + cb * p.bw, row_bytes, &full_bar[s]);
+                    const uint16_t *src = plane + tok * p.c + cb * p.bw;
+                    if (WIDE) {                                                 // the boxed stage layout, piece by piece
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            bulk_load(st + k * kBoxBytes + (size_t)lane * 2 * kBoxChannels, src + k * kBoxChannels,
+                                      2 * kBoxChannels, &full_bar[s]);
+                    } else {
+                        bulk_load(st + (size_t)lane * row_bytes, src, row_bytes, &full_bar[s]);
+                    }
                 }
             }
             ++unit;
