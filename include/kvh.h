@@ -204,7 +204,7 @@ kvh_status kvh_decode_batch(const void *streams_base, uint64_t streams_bytes,
  * pass -1 / -1 for any mix.  in_descs_host / out_descs_host [host, n_chunks each, may both be
  * NULL]: host copies of the two arrays; with them a mix is sorted by pair of levels on the host
  * and every pair runs through its specialised kernel (as kvh_encode_chunks does per level).  The
- * two stream buffers must not overlap.  n_channels <= 1024. */
+ * two stream buffers must not overlap.  Rows wider than 1024 channels: as for kvh_encode_kept. */
 kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, const kvh_chunk_desc *in_descs,
                          void *out_streams, uint64_t out_capacity, const kvh_chunk_desc *out_descs,
                          const kvh_chunk_desc *in_descs_host, const kvh_chunk_desc *out_descs_host,

@@ -30,8 +30,9 @@ auto pick_kernel(int lin, int lout) -> void (*)(const TranscodeParams, const int
 template <typename Chunks>
 kvh_status launch(const TranscodeParams &p, int lin, int lout, int n_chunks, cudaStream_t st, const Chunks &chunks)
 {
-    const unsigned grid = grid_for(n_chunks, p.l);
-    if (grid == 0) return KVH_ERR_BAD_SHAPE;
+    const int64_t tiles = (int64_t)grid_for(n_chunks, p.l) * p.n_blocks;
+    if (grid_for(n_chunks, p.l) == 0 || tiles > 0x7fffffffLL) return KVH_ERR_BAD_SHAPE;
+    const unsigned grid = (unsigned)tiles;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -59,7 +60,7 @@ extern "C" kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, c
     if (!in_streams || !out_streams || !in_descs || !out_descs || n_chunks < 0) return KVH_ERR_INVALID_ARG;
     const kvh_status s = check_shape(0, n_layers, n_channels);
     if (s != KVH_OK) return s;
-    if (n_channels > kEncMaxChannels) return KVH_ERR_BAD_SHAPE;      // a tile has to fit a shared-memory stage
+    if (block_width(n_channels) == 0) return KVH_ERR_BAD_SHAPE;      // a tile of a column block has to fit a stage
     if ((level_in < 0) != (level_out < 0)) return KVH_ERR_BAD_LEVEL;
     if (level_in >= 0 && (level_in >= kNumLevels || level_out >= kNumLevels || level_out <= level_in))
         return KVH_ERR_BAD_LEVEL;
@@ -76,6 +77,8 @@ extern "C" kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, c
     p.out_capacity = out_capacity;
     p.out_descs = out_descs;
     p.l = n_layers; p.c = n_channels;
+    p.bw = block_width(n_channels);
+    p.n_blocks = n_channels / p.bw;
     p.status = dev_status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (level_in >= 0 || !in_descs_host || !out_descs_host)

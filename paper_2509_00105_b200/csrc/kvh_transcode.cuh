@@ -31,6 +31,7 @@ struct TranscodeParams {
     uint64_t out_capacity;
     const kvh_chunk_desc *out_descs;    // device, n_chunks
     int32_t l, c;
+    int32_t bw, n_blocks;               // channels per column block (c when c <= 1024), blocks per row
     int32_t *status;
 };
 
@@ -94,11 +95,11 @@ __device__ __forceinline__ uint2 tc_row_k(const uint8_t *codes, const f32x2 (&lo
 }
 
 // K: a thread owns 4 channels and walks the tile's rows (any number of them).
-template <int BIN, int BOUT, int C>
-__device__ __forceinline__ void tc_consume_k(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+template <int BIN, int BOUT>
+__device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
                                              int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int c = C ? C : c_rt;
+    const int c = g.cw;                                  // channels per stage row
     if (tid < (c >> 2)) {
         const int cq = tid;
         const uint4 w4 = *reinterpret_cast<const uint4 *>(st + tc_meta_off(c) + 16 * (size_t)cq);
@@ -114,14 +115,17 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, int c_rt, int ti
             mask[i] = inv[i] != 0.0f ? 0xffffffffu : 0u;
             all_quantised = all_quantised && inv[i] != 0.0f;
         }
-        *reinterpret_cast<uint4 *>(meta_sec + 4 * ((size_t)tile * c + 4 * cq)) = make_uint4(m[0], m[1], m[2], m[3]);
+        uint4 *meta_out;
+        uint8_t *out;
+        uint32_t out_bytes;
+        enc_k_out<BOUT>(g, cq, tile, meta_sec, codes_sec, meta_out, out, out_bytes);
+        *meta_out = make_uint4(m[0], m[1], m[2], m[3]);
         const f32x2 lo[2] = {f2_make(l1[0], l1[1]), f2_make(l1[2], l1[3])};
         const f32x2 sc[2] = {f2_make(s1[0], s1[1]), f2_make(s1[2], s1[3])};
         const f32x2 lo_a = f2_make(lo_new[0], lo_new[1]), lo_b = f2_make(lo_new[2], lo_new[3]);
         const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
-        const uint32_t in_bytes = (uint32_t)c * BIN / 8, out_bytes = (uint32_t)c * BOUT / 8;
+        const uint32_t in_bytes = (uint32_t)c * BIN / 8;
         const uint8_t *src = st + (size_t)cq * BIN / 2;   // 4 codes = BIN / 2 bytes
-        uint8_t *out = codes_sec + ((size_t)tile * kTileTokens * c + 4 * cq) * BOUT / 8;
         if (all_quantised) {
 #pragma unroll 8
             for (int t = 0; t < nt; ++t)
@@ -138,17 +142,13 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, int c_rt, int ti
 }
 
 // V: a thread dequantises whole groups (32 codes, one metadata word) and encodes them again.
-template <int BIN, int BOUT, int C>
-__device__ __forceinline__ void tc_consume_v(const uint8_t *st, int c_rt, int tid, uint64_t *empty_bar,
+template <int BIN, int BOUT>
+__device__ __forceinline__ void tc_consume_v(const uint8_t *st, RowGeom geom, int tid, uint64_t *empty_bar,
                                              int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int c = C ? C : c_rt;
-    const int gpr = c >> 5;
-    const int ngroups = nt * gpr;
-    const uint32_t *meta_in = reinterpret_cast<const uint32_t *>(st + tc_meta_off(c));
-    const size_t g_first = (size_t)tile * kTileTokens * gpr;
-    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec) + g_first;
-    uint8_t *codes = codes_sec + g_first * (4 * BOUT);
+    const int ngroups = nt * (geom.cw >> 5);             // the tile's groups, in stage order
+    const uint32_t *meta_in = reinterpret_cast<const uint32_t *>(st + tc_meta_off(geom.cw));
+    uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec);
     const f32x2 pre01 = f2_make(Pos<BIN>::prescale(0), Pos<BIN>::prescale(1));
     const f32x2 pre23 = f2_make(Pos<BIN>::prescale(2), Pos<BIN>::prescale(3));
 #pragma unroll 2
@@ -166,7 +166,8 @@ __device__ __forceinline__ void tc_consume_v(const uint8_t *st, int c_rt, int ti
             spread8<BIN>(src + j * BIN, q);
             x[j] = fma_pack8(q, sc, lo);
         }
-        enc_group_v<BOUT, false>(x, 0, m, meta + g, codes + (size_t)g * (4 * BOUT));
+        const size_t gi = enc_v_group_index(geom, tile, g);
+        enc_group_v<BOUT, false>(x, 0, m, meta + gi, codes_sec + gi * (4 * BOUT));
     }
     enc_release(empty_bar);
 }
@@ -180,8 +181,9 @@ __device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_
         enc_consume_level<C, LOUT>(u, st, c_rt, tid, eb);            // raw rows: the encoder as it is
     } else {
         constexpr int BIN = 16 >> LIN, BOUT = 16 >> LOUT;
-        if (u.kv) tc_consume_v<BIN, BOUT, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
-        else tc_consume_k<BIN, BOUT, C>(st, c_rt, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        const RowGeom g = row_geom<C>(u.cw, c_rt, u.col0);
+        if (u.kv) tc_consume_v<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        else tc_consume_k<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
     }
 }
 template <int C, int LIN, int LOUT>
@@ -244,7 +246,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
 
     if (warp == kProducerWarp) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk;
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
         uint32_t unit = 0;
         bool ok = true;
         int cur_chunk = -1;
@@ -261,8 +263,10 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int tile = (int)(tile_id % kTilesPerChunk);
-            const int64_t plane_id = tile_id / kTilesPerChunk;
+            const int cb = (int)(tile_id % p.n_blocks);          // column block (rows wider than 1024 channels)
+            const int64_t row_tile = tile_id / p.n_blocks;
+            const int tile = (int)(row_tile % kTilesPerChunk);
+            const int64_t plane_id = row_tile / kTilesPerChunk;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), 0);
@@ -292,35 +296,51 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
             uint8_t *lay_out = p.out + dout.stream_off + (uint64_t)layer * Lo.layer_bytes();
             ok = acquire();
             if (!ok) return;
+            const int s = unit % kEncStages;
+            uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
+            const bool wide = p.n_blocks > 1;
+            const int col0 = cb * p.bw;
+            const uint32_t gpr = (uint32_t)p.c / kGroup;         // groups per plane row
+            const int b = level_bits(di.level);
+            // the block's codes (or raw rows) of row r: row_bytes at csrc + r * row_stride; its metadata: one
+            // piece of 4 * bw bytes for K, one piece of bw / 8 bytes per row for V
+            const uint8_t *csrc = lay_in + Li.codes_off(kv) + ((uint64_t)t0 * p.c + col0) * b / 8;
+            const uint32_t row_bytes = (uint32_t)p.bw * b / 8, row_stride = (uint32_t)p.c * b / 8;
+            const uint8_t *meta_in = lay_in + Li.meta_off(kv);
+            const uint8_t *msrc = kv == 0 ? meta_in + 4 * ((uint64_t)tile * p.c + col0)
+                                          : meta_in + 4 * ((uint64_t)t0 * gpr + col0 / kGroup);
+            const uint32_t mrow_bytes = 4u * (p.bw / kGroup), mrow_stride = 4u * gpr;
             if (lane == 0) {
-                const int s = unit % kEncStages;
                 TcUnit &u = info[s];
-                u.bits_in = level_bits(di.level);
+                u.bits_in = b;
                 u.e.bits = level_bits(dout.level); u.e.kv = kv; u.e.nt = nt; u.e.tile = tile;
-                u.e.last = t0 + nt == n;
+                u.e.last = t0 + nt == n && cb == p.n_blocks - 1;
                 u.e.meta_payload = (uint32_t)(kv ? Lo.vmeta_payload : Lo.kmeta_payload);
                 u.e.meta_padded = (uint32_t)(kv ? Lo.vmeta : Lo.kmeta);
                 u.e.codes_payload = (uint32_t)Lo.codes_payload;
                 u.e.codes_padded = (uint32_t)Lo.kcodes;
                 u.e.meta = lay_out + Lo.meta_off(kv);
                 u.e.codes = lay_out + Lo.codes_off(kv);
-                u.e.col0 = 0; u.e.cw = p.c;
-                uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
-                const uint8_t *codes_in = lay_in + Li.codes_off(kv);
-                if (di.level == 0) {
-                    const uint32_t bytes = 2u * (uint32_t)nt * (uint32_t)p.c;
-                    mbar_arrive_expect_tx(&full_bar[s], bytes);
-                    bulk_load(st, codes_in + 2 * (uint64_t)t0 * p.c, bytes, &full_bar[s]);
-                } else {
-                    const int b = level_bits(di.level);
-                    const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
-                    const uint8_t *meta_in = lay_in + Li.meta_off(kv);
-                    const uint8_t *msrc = kv == 0 ? meta_in + 4 * (uint64_t)tile * p.c
-                                                  : meta_in + 4 * (uint64_t)t0 * (p.c / kGroup);
-                    const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * (p.c / kGroup));
+                u.e.col0 = col0; u.e.cw = p.bw;
+                if (!wide) {
+                    const uint32_t cbytes = round16((uint32_t)nt * row_bytes);
+                    const uint32_t mbytes = di.level == 0 ? 0u : kv == 0 ? 4u * p.c : round16((uint32_t)nt * mrow_bytes);
                     mbar_arrive_expect_tx(&full_bar[s], cbytes + mbytes);
-                    bulk_load(st, codes_in + (uint64_t)t0 * p.c * b / 8, cbytes, &full_bar[s]);
-                    bulk_load(st + tc_meta_off(p.c), msrc, mbytes, &full_bar[s]);
+                    bulk_load(st, csrc, cbytes, &full_bar[s]);
+                    if (mbytes) bulk_load(st + tc_meta_off(p.bw), msrc, mbytes, &full_bar[s]);
+                } else {
+                    const uint32_t mbytes = di.level == 0 ? 0u : kv == 0 ? 4u * p.bw : (uint32_t)nt * mrow_bytes;
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nt * row_bytes + mbytes);
+                    if (di.level != 0 && kv == 0) bulk_load(st + tc_meta_off(p.bw), msrc, 4u * p.bw, &full_bar[s]);
+                }
+            }
+            if (wide) {                                  // lane r copies row r's pieces (the expectation is posted first)
+                __syncwarp();
+                if (lane < nt) {
+                    bulk_load(st + (size_t)lane * row_bytes, csrc + (size_t)lane * row_stride, row_bytes, &full_bar[s]);
+                    if (di.level != 0 && kv == 1)
+                        bulk_load(st + tc_meta_off(p.bw) + (size_t)lane * mrow_bytes, msrc + (size_t)lane * mrow_stride,
+                                  mrow_bytes, &full_bar[s]);
                 }
             }
             ++unit;

@@ -48,7 +48,8 @@ def run_case(kvh, l, c, N, levels_in, levels_out, hint):
         assert np.array_equal(g[:total], want) and np.all(g[total:] == 0xAB)
 
 
-@pytest.mark.parametrize("l,c,N", [(1, 1024, 300), (2, 256, 257), (1, 32, 33), (1, 96, 700), (2, 1024, 64)])
+@pytest.mark.parametrize("l,c,N", [(1, 1024, 300), (2, 256, 257), (1, 32, 33), (1, 96, 700), (2, 1024, 64),
+                                   (1, 2048, 70), (1, 1152, 40)])
 @pytest.mark.parametrize("pair", PAIRS)
 def test_transcode_one_pair_of_levels(kvh, l, c, N, pair):
     run_case(kvh, l, c, N, pair[0], pair[1], pair)       # the kernel specialised for the pair

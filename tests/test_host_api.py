@@ -163,7 +163,7 @@ def test_launches_too_large_for_a_grid_and_new_entry_points_reject_before_any_cu
     assert L.kvh_transcode(None, 4096, a, a, 4096, a, None, None, 1, 1, 32, -1, -1, None, None) == 1
     assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 32, 2, 1, None, None) == 2
     assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 32, 1, -1, None, None) == 2
-    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 2048, 0, 1, None, None) == 3
+    assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 1, 1, 2080, 0, 1, None, None) == 3
     assert L.kvh_transcode(a + 64, 4096, a, a, 4096, a, None, None, 1, 1, 32, 0, 1, None, None) == 4
     assert L.kvh_transcode(a, 4096, a, a, 4096, a, None, None, 0, 1, 32, 0, 1, None, None) == 0      # nothing to do
     # token dropping: runs
