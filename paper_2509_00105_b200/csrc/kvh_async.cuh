@@ -93,4 +93,55 @@ __device__ __forceinline__ bool clc_query(const void *response, uint32_t &ctaid_
     return valid != 0;
 }
 
+// The tiles a persistent CTA works through, as seen by its producer warp (all 32 lanes call every
+// member).  sched 0: blockIdx.x, blockIdx.x + gridDim.x, ...  sched 1: the grid holds one CTA per
+// tile; a CTA starts with its own index and then takes over CTAs that have not started yet, asking
+// for the next one (ask) before it feeds the current tile so that the answer is there when needed.
+struct TileFeed {
+    uint4 *response;               // shared: 2 answers
+    uint64_t *bar;                 // shared: 2 mbarriers, initialised with count 1
+    int sched, lane;
+    volatile int *abort_flag;
+    uint32_t query = 0;            // answers asked for so far
+    bool asked = false;            // one answer still outstanding
+
+    __device__ __forceinline__ void ask()
+    {
+        if (sched != 1) return;
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&bar[query & 1], 16);
+            clc_try_cancel(&response[query & 1], &bar[query & 1]);
+        }
+        asked = true;
+    }
+    // Moves tile_id on.  1: there is a next tile; 0: none left; -1: the wait for the answer ran out.
+    __device__ __forceinline__ int next(int64_t &tile_id, int64_t total_tiles)
+    {
+        if (sched != 1) {
+            tile_id += gridDim.x;
+            return tile_id < total_tiles ? 1 : 0;
+        }
+        uint32_t got = 0, id = 0, w = 1;
+        if (lane == 0) {
+            w = mbar_wait(&bar[query & 1], (query >> 1) & 1, abort_flag);
+            if (w) got = clc_query(&response[query & 1], id);
+        }
+        w = __shfl_sync(0xffffffffu, w, 0);
+        got = __shfl_sync(0xffffffffu, got, 0);
+        id = __shfl_sync(0xffffffffu, id, 0);
+        if (!w) return -1;
+        asked = false;
+        ++query;
+        if (!got) return 0;                              // no CTA left to take over: never ask again
+        tile_id = id;
+        return tile_id < total_tiles ? 1 : 0;
+    }
+    // Before the CTA leaves: an answer still on its way has to land (lane 0).
+    __device__ __forceinline__ void drain()
+    {
+        int never = 0;
+        if (asked) (void)mbar_wait(&bar[query & 1], (query >> 1) & 1, &never);
+    }
+};
+
 }  // namespace kvh

@@ -383,36 +383,15 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             }
         };
 
+        TileFeed feed{clc_response, clc_bar, sched, lane, &abort_flag};
         int64_t tile_id = blockIdx.x;
-        uint32_t query = 0;                              // answers asked for so far
-        bool asked = false;                              // one answer still outstanding
         while (ok && tile_id < total_tiles) {
-            if (sched == 1) {                            // ask for the next tile while this one streams
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(&clc_bar[query & 1], 16);
-                    clc_try_cancel(&clc_response[query & 1], &clc_bar[query & 1]);
-                }
-                asked = true;
-            }
+            feed.ask();                                  // the next tile's index travels while this one streams
             do_tile(tile_id);
             if (!ok) break;
-            if (sched == 1) {
-                uint32_t got = 0, next = 0, w = 1;
-                if (lane == 0) {
-                    w = mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &abort_flag);
-                    if (w) got = clc_query(&clc_response[query & 1], next);
-                }
-                w = __shfl_sync(0xffffffffu, w, 0);
-                got = __shfl_sync(0xffffffffu, got, 0);
-                next = __shfl_sync(0xffffffffu, next, 0);
-                if (!w) { ok = false; break; }
-                asked = false;
-                ++query;
-                if (!got) break;                         // no CTA left to take over: never ask again
-                tile_id = next;
-            } else {
-                tile_id += gridDim.x;
-            }
+            const int more = feed.next(tile_id, total_tiles);
+            if (more < 0) ok = false;
+            if (more <= 0) break;
         }
         if (ok) ok = emit(0, 0, 0, 0, nullptr, 0, nullptr, 0, 0, nullptr, 0, 0);      // end marker
         if (!ok && lane == 0) {
@@ -426,7 +405,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const uint32_t first = unit > (uint32_t)n_stages ? unit - n_stages : 0;
             for (uint32_t w = first; w < unit; ++w)
                 (void)mbar_wait(&full_bar[w % n_stages], (w / n_stages) & 1, &never);
-            if (asked) (void)mbar_wait(&clc_bar[query & 1], (query >> 1) & 1, &never);
+            feed.drain();
         }
     } else {
         // ------------------------------ consumer warps ------------------------------
