@@ -9,6 +9,10 @@
 namespace kvh {
 
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: no wait in a kernel lasts longer
+// How long one try_wait may keep its warp suspended in hardware before it reports "not yet": a
+// waiting warp then costs a few instructions per microsecond instead of a busy loop that competes
+// with the working warps for issue slots.  The wait still ends the moment the phase completes.
+constexpr uint32_t kTryWaitHintNs = 20000u;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -29,9 +33,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity), "r"(kTryWaitHintNs) : "memory");
     return done != 0;
 }
 __device__ __forceinline__ unsigned long long global_ns()
