@@ -20,7 +20,7 @@
  *     macros N, c, l, k).
  * The design section that would define the levels is not part of the paper's
  * text, so the level ladder, group geometry, metadata and bit order below are
- * this build's stated reading of it.  PARITY UNPINNED against the paper's own
+ * this library's stated reading of it.  PARITY UNPINNED against the paper's own
  * quantiser parameters (group size, metadata format): nothing printed in the
  * paper can confirm or refute them.  Everything else is pinned by the CPU
  * tests (closed forms, a hand-worked group, invariants, an independent

@@ -114,7 +114,7 @@ def test_paper_capacity_example():
     # "millions of tokens" <-> 3 TB of KV
     assert g["agentic_kv_bytes"] / per_token > g["agentic_tokens_at_least"]
     assert g["agentic_kv_bytes"] / per_token < 20e6
-    # the 32768-token 70B-shaped context of the benchmark definition is ~10.7 GB
+    # the 32768-token 70B-shaped context of the benchmark is ~10.7 GB
     assert abs(128 * oracle.level_bytes(0, 80, 1024, 256) / 1e9 - 10.7) < 0.05
 
 

@@ -28,7 +28,7 @@ class Shape:
     n_tokens: int
 
 
-# The five workloads the benchmark definition names (index = config number - 1).
+# The shapes of the five benchmark workloads.
 TINY = Shape("tiny", 4, 1024, 256)
 LLAMA8B_8K = Shape("llama3-8b-8k", 32, 1024, 8192)
 LLAMA70B_32K = Shape("llama3-70b-32k", 80, 1024, 32768)
