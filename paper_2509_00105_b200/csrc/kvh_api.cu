@@ -90,7 +90,7 @@ bool make_kv_map(const EncodeParams &p, CUtensorMap *map)
     const cuuint64_t strides[1] = {(cuuint64_t)p.c * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kBoxChannels, (cuuint32_t)kTileTokens};
     const cuuint32_t elem[2] = {1, 1};
-    if (dims[1] > 0xffffffffull) return false;
+    if (dims[1] > 0x7fffffffull) return false;           // row coordinates are 32-bit signed
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<uint16_t *>(p.kv), dims, strides, box, elem,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
