@@ -70,9 +70,6 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     return launch_status();
 }
 
-// Encode launch: the persistent TMA-fed kernel when a 32-token tile fits a shared-memory stage,
-// otherwise one CTA per tile reading global memory directly.  KVH_ENCODE_PATH=direct forces the
-// latter and KVH_ENCODE_SCHED=static a fixed tile stride (measurement aids).
 // Tensor map of the encode source seen as a 2-D tensor [n_layers * 2 * src_N rows][c channels] of
 // bf16, with boxes of 256 channels x 32 rows; false if the driver entry point is not to be had.
 bool make_kv_map(const EncodeParams &p, CUtensorMap *map)
@@ -132,6 +129,10 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
     return launch_status();
 }
 
+// Encode launch: the persistent TMA-fed kernel when rows are at most 1024 channels wide or divide
+// into column blocks, otherwise one CTA per tile reading global memory directly.
+// KVH_ENCODE_PATH=direct forces the latter and KVH_ENCODE_SCHED=static a fixed tile stride
+// (measurement aids).
 // descs_host (may be nullptr): the caller's host copy of p.descs, indexed like it.  With it the
 // chunks of each level go, as index lists in the kernel parameters, to the instance specialised for
 // that level; without it one instance that holds all levels takes the chunks in order.
