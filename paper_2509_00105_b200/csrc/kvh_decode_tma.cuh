@@ -1,4 +1,5 @@
-// Persistent, TMA-fed decode kernel (the fast path for c <= 1024, pages of >= 16 tokens).
+// Persistent, TMA-fed decode kernel (pages of >= 16 tokens; rows of up to 1024 channels, or wider
+// rows that divide into equal column blocks, which are fed with one bulk copy per row).
 //
 // One CTA (or a few) per SM loops over work units.  A producer warp walks the CTA's share of
 // (chunk, layer, K|V, 32-token tile) tiles, resolves descriptors and page ids, and streams each

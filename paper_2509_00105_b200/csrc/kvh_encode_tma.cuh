@@ -1,4 +1,4 @@
-// Persistent, TMA-fed encode kernel (the fast path for c <= 1024).
+// Persistent, TMA-fed encode kernel.
 //
 // Storing a context is the executor's other direction: the policy has decided to keep an entry
 // "in full quality" (level 0) or to compress it (levels 1..3), and the KV tensor has to be turned
@@ -17,6 +17,11 @@
 // packed binary32 instructions of sm_100 (sub/mul/fma .rn.f32x2: IEEE round-to-nearest on each
 // half, no flush to zero), which halves the issue slots the arithmetic takes.  A stage is handed
 // back to the producer as soon as its data sits in registers.
+//
+// Rows wider than 1024 channels are cut into column blocks (RowGeom): blocks of 1024 channels come
+// in through 2-D tiled TMA (a tensor map over the source, four boxes of 256 channels x 32 rows per
+// tile), other widths and token dropping (kept runs gathered into a compact sequence) through one
+// 1-D bulk copy per row issued by the producer's lanes in parallel.
 //
 // Tiles are handed out dynamically through cluster launch control, as in the decode kernel.  Every
 // wait is bounded: when one runs out the CTA reports KVH_ERR_TIMEOUT, raises its abort flag,
