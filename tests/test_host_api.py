@@ -181,3 +181,16 @@ def test_launches_too_large_for_a_grid_and_new_entry_points_reject_before_any_cu
     choice = np.zeros(1, dtype=np.int32)
     assert L.kvh_policy_assign(freq.ctypes.data, opts.ctypes.data, begin.ctypes.data, 1, tier.ctypes.data,
                                choice.ctypes.data, None, None) == 1
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/kvh.h is a C header: a C99 compiler takes it with warnings as errors."""
+    import subprocess
+    src = tmp_path / "use_kvh.c"
+    src.write_text('#include "kvh.h"\n'
+                   "int main(void) { kvh_token_run r = {0, 1}; kvh_option o = {1, 0.5}; kvh_tier t = {1.0, 1.0, 1};\n"
+                   "  kvh_pool p; kvh_chunk_desc d; (void)r; (void)o; (void)t; (void)p; (void)d;\n"
+                   "  return kvh_format_version() == KVH_FORMAT_VERSION ? 0 : 1; }\n")
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", f"-I{inc}", str(src)],
+                   check=True)
