@@ -36,13 +36,13 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     const unsigned grid = grid_for(n_chunks, p.l);
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
     // KVH_DECODE_PATH=direct forces the one-CTA-per-tile kernel (a measurement aid); the
-    // persistent TMA kernel needs a tile to fit a shared-memory stage and at most 2 pages per tile.
+    // persistent TMA kernel needs a column block to fit a shared-memory stage and pages of at least 8 tokens.
     const char *force = getenv("KVH_DECODE_PATH");
     const bool want_tma = !(force && strcmp(force, "direct") == 0);
     p.bw = block_width(p.c);                             // rows wider than 1024 channels go in column blocks
     p.n_blocks = p.bw > 0 ? p.c / p.bw : 1;
     const int64_t tiles = (int64_t)grid * p.n_blocks;
-    if (want_tma && p.bw > 0 && tiles <= 0x7fffffffLL && p.page_tokens >= 16) {
+    if (want_tma && p.bw > 0 && tiles <= 0x7fffffffLL && p.page_tokens >= 8) {    // a lane per page id of a chunk
         int dev = 0, sms = 0, per_sm = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)

@@ -1,4 +1,4 @@
-// Persistent, TMA-fed decode kernel (pages of >= 16 tokens; rows of up to 1024 channels, or wider
+// Persistent, TMA-fed decode kernel (pages of >= 8 tokens; rows of up to 1024 channels, or wider
 // rows that divide into equal column blocks, which are fed with one bulk copy per row).
 //
 // One CTA (or a few) per SM loops over work units.  A producer warp walks the CTA's share of
@@ -32,7 +32,7 @@ struct UnitInfo {
     int32_t kv;          // 0 K, 1 V
     int32_t row0;        // first token of the unit within its chunk
     int32_t nrows;       // tokens in the unit (1..32)
-    int32_t pg0, pg1;    // page ids of the page holding row0 and of the next one
+    int32_t pg[4];       // page ids of the page holding row0 and of the next three (pages hold >= 8 tokens)
     uint16_t *plane;     // pool + layer*layer_stride + kv*kv_stride
     int32_t col0, cw;    // first channel and width of the unit's column block (0, c unless rows exceed 1024 channels)
 };
@@ -112,29 +112,45 @@ __device__ __forceinline__ uint4 fma_pack8(const f32x2 (&x)[4], const f32x2 (&sc
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Rows of a unit are dealt to threads in runs of `rpt` consecutive rows (a power of two, so a run
-// never straddles a page); `cv` is the thread's 8-channel vector within the row.
+// Rows of a unit are dealt to threads in runs of consecutive rows: `rpt` rows per thread (a power of
+// two: 16 when c = 1024), cut into runs of at most a page, so that a run never straddles a page;
+// `cv` is the thread's 8-channel vector within the row.
 struct RowRun {
     int cv, first, count;       // count == 0 for idle threads
     uint16_t *dst;              // first row's destination (already offset by cv), nullptr if none
 };
+struct RowRuns {
+    int cv, g, rpp, len, n;     // thread's vector and row group; row groups; rows per run; runs per thread
+};
 
 template <int C>
-__device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u)
+__device__ __forceinline__ RowRuns row_runs(const DecodeParams &p, const UnitInfo &u)
 {
     const int V8 = (C ? C : u.cw) >> 3;                   // 16-byte vectors per stage row, <= 128
-    const int rpp = kConsumerThreads / V8;                // row groups the CTA holds, >= 2
+    RowRuns rr;
+    rr.rpp = kConsumerThreads / V8;                       // row groups the CTA holds, >= 2
     int rpt = 1;
-    while (rpt * rpp < kTileTokens) rpt <<= 1;            // rows per thread: 16 when c = 1024
-    const int g = threadIdx.x / V8;
+    while (rpt * rr.rpp < kTileTokens) rpt <<= 1;         // rows per thread
+    rr.len = min(rpt, p.page_tokens);
+    rr.n = rpt / rr.len;
+    rr.g = threadIdx.x / V8;
+    rr.cv = threadIdx.x - rr.g * V8;
+    return rr;
+}
+
+// Run i of the thread: rows [first, first + count) of the unit.
+template <int C>
+__device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u, const RowRuns &rr, int i)
+{
     RowRun r;
-    r.cv = threadIdx.x - g * V8;
-    r.first = g * rpt;
-    r.count = g < rpp ? max(0, min(rpt, u.nrows - r.first)) : 0;
+    r.cv = rr.cv;
+    r.first = (i * rr.rpp + rr.g) * rr.len;
+    r.count = rr.g < rr.rpp ? max(0, min(rr.len, u.nrows - r.first)) : 0;
     r.dst = nullptr;
     if (r.count > 0) {
         const int T = u.row0 + r.first;
-        const int32_t pg = (T >> p.page_shift) == (u.row0 >> p.page_shift) ? u.pg0 : u.pg1;
+        const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);      // 0..3; selects keep u in registers
+        const int32_t pg = pi == 0 ? u.pg[0] : pi == 1 ? u.pg[1] : pi == 2 ? u.pg[2] : u.pg[3];
         r.dst = page_row<C>(p, pg, u.plane, T);              // reports an out-of-range page id
         if (r.dst) r.dst += (C ? 0 : u.col0) + 8 * r.cv; else r.count = 0;
     }
@@ -145,12 +161,15 @@ template <int C>
 __device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
 {
     const int cw = C ? C : u.cw;                          // row width in the stage
-    const RowRun r = row_run<C>(p, u);
-    const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * cw + 8 * r.cv));
-    uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
     const int sstride = cw >> 3, dstride = (C ? C : p.c) >> 3;    // uint4 per stage row / per page row
+    const RowRuns rr = row_runs<C>(p, u);
+    for (int i = 0; i < rr.n; ++i) {
+        const RowRun r = row_run<C>(p, u, rr, i);
+        const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * cw + 8 * r.cv));
+        uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
 #pragma unroll 4
-    for (int k = 0; k < r.count; ++k) dst[(size_t)k * dstride] = src[(size_t)k * sstride];
+        for (int k = 0; k < r.count; ++k) dst[(size_t)k * dstride] = src[(size_t)k * sstride];
+    }
 }
 
 template <int BITS, int C>
@@ -159,11 +178,11 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
 {
     const int c = C ? C : u.cw;                           // row width in the stage
     const int dstride = C ? C : p.c;                      // row width of a page
-    const RowRun r = row_run<C>(p, u);
-    if (r.count == 0) return;
+    const RowRuns rr = row_runs<C>(p, u);
+    if (rr.g >= rr.rpp) return;
     f32x2 lo[4], sc[4];
     {
-        const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * r.cv;
+        const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * rr.cv;
         const uint4 m0 = m[0], m1 = m[1];
         const uint32_t w[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
         float l1[8], s1[8];
@@ -179,15 +198,18 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
         }
     }
     const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-    const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
-    uint16_t *dst = r.dst;
+    for (int i = 0; i < rr.n; ++i) {
+        const RowRun r = row_run<C>(p, u, rr, i);
+        const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
+        uint16_t *dst = r.dst;
 #pragma unroll 4
-    for (int k = 0; k < r.count; ++k) {
-        f32x2 x[4];
-        spread8<BITS>(src, x);
-        *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
-        src += row_bytes;
-        dst += dstride;
+        for (int k = 0; k < r.count; ++k) {
+            f32x2 x[4];
+            spread8<BITS>(src, x);
+            *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
+            src += row_bytes;
+            dst += dstride;
+        }
     }
 }
 
@@ -197,38 +219,41 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
 {
     const int c = C ? C : u.cw;                           // row width in the stage
     const int dstride = C ? C : p.c;                      // row width of a page
-    const RowRun r = row_run<C>(p, u);
+    const RowRuns rr = row_runs<C>(p, u);
     const int lane = threadIdx.x & 31;
     const uint32_t quad = 0xfu << (lane & ~3);            // the 4 lanes that share every V group
     const int groups = c / kGroup;
-    const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)r.first * groups + (r.cv >> 2);
     const uint32_t row_bytes = (uint32_t)c * BITS / 8;
-    const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
-    uint16_t *dst = r.dst;
     const f32x2 pre01 = f2_make(Pos<BITS>::prescale(0), Pos<BITS>::prescale(1));
     const f32x2 pre23 = f2_make(Pos<BITS>::prescale(2), Pos<BITS>::prescale(3));
-    // r.count is the same for the 4 lanes of a quad (they share the row group), so the shuffles
-    // below are executed by whole quads
-    for (int kb = 0; kb < r.count; kb += 4) {
-        // each lane of the quad derives the scale of one of the next 4 rows: a quarter of a
-        // division per row and lane
-        float mine = 0.0f, unused;
-        const int kq = kb + (lane & 3);
-        if (kq < r.count) decode_params<BITS>(mrow[(size_t)kq * groups], unused, mine);
+    for (int i = 0; i < rr.n; ++i) {
+        const RowRun r = row_run<C>(p, u, rr, i);
+        const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)r.first * groups + (r.cv >> 2);
+        const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
+        uint16_t *dst = r.dst;
+        // r.count is the same for the 4 lanes of a quad (they share the row group and the page), so
+        // the shuffles below are executed by whole quads
+        for (int kb = 0; kb < r.count; kb += 4) {
+            // each lane of the quad derives the scale of one of the next 4 rows: a quarter of a
+            // division per row and lane
+            float mine = 0.0f, unused;
+            const int kq = kb + (lane & 3);
+            if (kq < r.count) decode_params<BITS>(mrow[(size_t)kq * groups], unused, mine);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (kb + j < r.count) {
-                const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
-                const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
-                const f32x2 ss = f2_make(s0, s0);
-                const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);      // exact: powers of two
-                const f32x2 ll = f2_make(l1, l1);
-                const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
-                f32x2 x[4];
-                spread8<BITS>(src, x);
-                *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
-                src += row_bytes;
-                dst += dstride;
+            for (int j = 0; j < 4; ++j) {
+                if (kb + j < r.count) {
+                    const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
+                    const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
+                    const f32x2 ss = f2_make(s0, s0);
+                    const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);      // exact: powers of two
+                    const f32x2 ll = f2_make(l1, l1);
+                    const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+                    f32x2 x[4];
+                    spread8<BITS>(src, x);
+                    *reinterpret_cast<uint4 *>(dst) = fma_pack8(x, sc, lo);
+                    src += row_bytes;
+                    dst += dstride;
+                }
             }
         }
     }
@@ -291,13 +316,15 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                 if (!w) return false;
             }
             const int pidx = row0 >> p.page_shift;
-            const int32_t pg0 = __shfl_sync(0xffffffffu, my_pg, pidx & 31);
-            const int32_t pg1 = __shfl_sync(0xffffffffu, my_pg, (pidx + 1) & 31);
+            int32_t pg[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) pg[i] = __shfl_sync(0xffffffffu, my_pg, (pidx + i) & 31);
             uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const bool strided = row_stride != 0;
             if (lane == 0) {
                 UnitInfo &u = info[s];
-                u.bits = bits; u.kv = kv; u.row0 = row0; u.nrows = nrows; u.pg0 = pg0; u.pg1 = pg1; u.plane = plane;
+                u.bits = bits; u.kv = kv; u.row0 = row0; u.nrows = nrows; u.plane = plane;
+                u.pg[0] = pg[0]; u.pg[1] = pg[1]; u.pg[2] = pg[2]; u.pg[3] = pg[3];
                 u.col0 = col0; u.cw = p.bw;
                 if (bits == 0) {
                     mbar_arrive(&full_bar[s]);

@@ -260,20 +260,32 @@ def test_bad_descriptors_are_skipped_and_reported(kvh):
     assert np.all(out3.cpu().numpy()[offsets[1]:] == 0xEE)
 
 
-def test_page_size_other_than_16(kvh):
-    l, c, N = 1, 64, 100
+@pytest.mark.parametrize("path", ["default", "direct"])
+@pytest.mark.parametrize("l,c,N", [(1, 64, 100), (2, 1024, 300), (1, 2048, 77)])
+def test_page_size_other_than_16(kvh, monkeypatch, l, c, N, path):
+    """Pages of 8 tokens and more go through the persistent kernel (a thread's run of rows is cut at
+    page boundaries: a 32-token tile then spans up to 4 pages); smaller pages take the direct one."""
+    if path == "direct":
+        monkeypatch.setenv("KVH_DECODE_PATH", "direct")
+    else:
+        monkeypatch.delenv("KVH_DECODE_PATH", raising=False)
     kv = workloads.make_kv(l, N, c, seed=12, device="cuda")
-    for page_tokens in (8, 32, 64):
-        for level in (0, 3):
+    for page_tokens in (4, 8, 32, 64, 256):
+        for level in (0, 1, 3):
             got, _ = kvh.encode(kv, level)
             want, offsets = oracle.encode_context(to_np16(kv), level)
-            npg = -(-N // page_tokens)
-            ids = torch.randperm(npg + 2, generator=torch.Generator().manual_seed(3))[:npg].to(torch.int32)
-            flat, view, strides = sentinel_pool(l, npg + 2, c, page_tokens=page_tokens)
-            kvh.decode_to_pages(got, level, N, ids.cuda(), kvh.Pool(view))
-            wp, _ = oracle_pool(flat.numel(), strides, want, offsets, [N], [level], l, c, ids.numpy(), npg + 2,
+            per_chunk = 256 // page_tokens
+            n_chunks = workloads.n_chunks(N)
+            ids = torch.randperm(n_chunks * per_chunk + 2, generator=torch.Generator().manual_seed(3))[:n_chunks * per_chunk].to(torch.int32)
+            flat, view, strides = sentinel_pool(l, n_chunks * per_chunk + 2, c, page_tokens=page_tokens)
+            descs, _ = kvh.plan_chunks(l, c, N, level, page_tokens=page_tokens)
+            status = new_status()
+            kvh.decode_batch(got, kvh.descs_to_tensor(descs, "cuda"), n_chunks, ids.cuda(), kvh.Pool(view), status)
+            ntoks, lv, _ = oracle.chunk_plan(N, level, l, c)
+            wp, _ = oracle_pool(flat.numel(), strides, want, offsets, ntoks, lv, l, c, ids.numpy(), n_chunks * per_chunk + 2,
                                 page_tokens)
-            assert np.array_equal(to_np16(flat), wp)
+            assert status.item() == 0
+            assert np.array_equal(to_np16(flat), wp), f"page_tokens {page_tokens} level {level}"
 
 
 def test_gpu_decodes_oracle_streams_and_oracle_decodes_gpu_streams(kvh):
