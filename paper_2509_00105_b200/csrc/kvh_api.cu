@@ -52,7 +52,9 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
         const size_t dyn = (size_t)stages * stage;
         // the instance with the channel count of the Llama-3 shapes compiled in, or the general one
-        auto kernel = p.c == 1024 ? decode_tma_kernel<1024> : decode_tma_kernel<0>;
+        const bool small_pages = p.page_tokens < 16;       // a thread's rows may then span several pages
+        auto kernel = p.c == 1024 ? (small_pages ? decode_tma_kernel<1024, true> : decode_tma_kernel<1024, false>)
+                                  : (small_pages ? decode_tma_kernel<0, true> : decode_tma_kernel<0, false>);
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kTmaThreads, dyn) != cudaSuccess ||
             per_sm < 1)

@@ -123,7 +123,9 @@ struct RowRuns {
     int cv, g, rpp, len, n;     // thread's vector and row group; row groups; rows per run; runs per thread
 };
 
-template <int C>
+// SMALLPG: pages may hold fewer tokens than a thread has rows (8-token pages); otherwise a thread
+// has one run and a tile at most two pages, which the compiler then knows.
+template <int C, bool SMALLPG>
 __device__ __forceinline__ RowRuns row_runs(const DecodeParams &p, const UnitInfo &u)
 {
     const int V8 = (C ? C : u.cw) >> 3;                   // 16-byte vectors per stage row, <= 128
@@ -131,15 +133,15 @@ __device__ __forceinline__ RowRuns row_runs(const DecodeParams &p, const UnitInf
     rr.rpp = kConsumerThreads / V8;                       // row groups the CTA holds, >= 2
     int rpt = 1;
     while (rpt * rr.rpp < kTileTokens) rpt <<= 1;         // rows per thread
-    rr.len = min(rpt, p.page_tokens);
-    rr.n = rpt / rr.len;
+    rr.len = SMALLPG ? min(rpt, p.page_tokens) : rpt;
+    rr.n = SMALLPG ? rpt / rr.len : 1;
     rr.g = threadIdx.x / V8;
     rr.cv = threadIdx.x - rr.g * V8;
     return rr;
 }
 
 // Run i of the thread: rows [first, first + count) of the unit.
-template <int C>
+template <int C, bool SMALLPG>
 __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo &u, const RowRuns &rr, int i)
 {
     RowRun r;
@@ -150,21 +152,21 @@ __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo 
     if (r.count > 0) {
         const int T = u.row0 + r.first;
         const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);      // 0..3; selects keep u in registers
-        const int32_t pg = pi == 0 ? u.pg[0] : pi == 1 ? u.pg[1] : pi == 2 ? u.pg[2] : u.pg[3];
+        const int32_t pg = pi == 0 ? u.pg[0] : (!SMALLPG || pi == 1) ? u.pg[1] : pi == 2 ? u.pg[2] : u.pg[3];
         r.dst = page_row<C>(p, pg, u.plane, T);              // reports an out-of-range page id
         if (r.dst) r.dst += (C ? 0 : u.col0) + 8 * r.cv; else r.count = 0;
     }
     return r;
 }
 
-template <int C>
+template <int C, bool SMALLPG>
 __device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
 {
     const int cw = C ? C : u.cw;                          // row width in the stage
     const int sstride = cw >> 3, dstride = (C ? C : p.c) >> 3;    // uint4 per stage row / per page row
-    const RowRuns rr = row_runs<C>(p, u);
+    const RowRuns rr = row_runs<C, SMALLPG>(p, u);
     for (int i = 0; i < rr.n; ++i) {
-        const RowRun r = row_run<C>(p, u, rr, i);
+        const RowRun r = row_run<C, SMALLPG>(p, u, rr, i);
         const uint4 *src = reinterpret_cast<const uint4 *>(codes + 2 * ((size_t)r.first * cw + 8 * r.cv));
         uint4 *dst = reinterpret_cast<uint4 *>(r.dst);
 #pragma unroll 4
@@ -172,13 +174,13 @@ __device__ __forceinline__ void consume_raw(const DecodeParams &p, const UnitInf
     }
 }
 
-template <int BITS, int C>
+template <int BITS, int C, bool SMALLPG>
 __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
     const int c = C ? C : u.cw;                           // row width in the stage
     const int dstride = C ? C : p.c;                      // row width of a page
-    const RowRuns rr = row_runs<C>(p, u);
+    const RowRuns rr = row_runs<C, SMALLPG>(p, u);
     if (rr.g >= rr.rpp) return;
     f32x2 lo[4], sc[4];
     {
@@ -199,7 +201,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     }
     const uint32_t row_bytes = (uint32_t)c * BITS / 8;
     for (int i = 0; i < rr.n; ++i) {
-        const RowRun r = row_run<C>(p, u, rr, i);
+        const RowRun r = row_run<C, SMALLPG>(p, u, rr, i);
         const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
         uint16_t *dst = r.dst;
 #pragma unroll 4
@@ -213,13 +215,13 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     }
 }
 
-template <int BITS, int C>
+template <int BITS, int C, bool SMALLPG>
 __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
                                           const uint8_t *meta)
 {
     const int c = C ? C : u.cw;                           // row width in the stage
     const int dstride = C ? C : p.c;                      // row width of a page
-    const RowRuns rr = row_runs<C>(p, u);
+    const RowRuns rr = row_runs<C, SMALLPG>(p, u);
     const int lane = threadIdx.x & 31;
     const uint32_t quad = 0xfu << (lane & ~3);            // the 4 lanes that share every V group
     const int groups = c / kGroup;
@@ -227,7 +229,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
     const f32x2 pre01 = f2_make(Pos<BITS>::prescale(0), Pos<BITS>::prescale(1));
     const f32x2 pre23 = f2_make(Pos<BITS>::prescale(2), Pos<BITS>::prescale(3));
     for (int i = 0; i < rr.n; ++i) {
-        const RowRun r = row_run<C>(p, u, rr, i);
+        const RowRun r = row_run<C, SMALLPG>(p, u, rr, i);
         const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)r.first * groups + (r.cv >> 2);
         const uint8_t *src = codes + (size_t)r.first * row_bytes + (size_t)r.cv * BITS;
         uint16_t *dst = r.dst;
@@ -262,7 +264,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
 // sched: 0 = each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... (grid = resident CTAs);
 //        1 = grid holds one CTA per tile and running CTAs pull further tiles through cluster
 //            launch control, so faster SMs take more tiles.
-template <int C>
+template <int C, bool SMALLPG = false>
 __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodeParams p, const int n_chunks,
                                                                  const int n_stages, const int sched)
 {
@@ -449,13 +451,13 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const uint8_t *mt = st + meta_off;
             switch (u.bits * 2 + u.kv) {                      // uniform per CTA
-            case 32: case 33: consume_raw<C>(p, u, st); break;
-            case 16: consume_k<8, C>(p, u, st, mt); break;
-            case 17: consume_v<8, C>(p, u, st, mt); break;
-            case 8: consume_k<4, C>(p, u, st, mt); break;
-            case 9: consume_v<4, C>(p, u, st, mt); break;
-            case 4: consume_k<2, C>(p, u, st, mt); break;
-            default: consume_v<2, C>(p, u, st, mt); break;
+            case 32: case 33: consume_raw<C, SMALLPG>(p, u, st); break;
+            case 16: consume_k<8, C, SMALLPG>(p, u, st, mt); break;
+            case 17: consume_v<8, C, SMALLPG>(p, u, st, mt); break;
+            case 8: consume_k<4, C, SMALLPG>(p, u, st, mt); break;
+            case 9: consume_v<4, C, SMALLPG>(p, u, st, mt); break;
+            case 4: consume_k<2, C, SMALLPG>(p, u, st, mt); break;
+            default: consume_v<2, C, SMALLPG>(p, u, st, mt); break;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[s]);
