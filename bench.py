@@ -409,7 +409,10 @@ def run_ours(args, shape: workloads.Shape):
         cores = len(os.sched_getaffinity(0))
         kv_np, layers = oracle_inputs(shape, cores, target_s=4.0)
         e, d, el = oracle_sample_step(kv_np, cores)
+        one_np = np.ascontiguousarray(kv_np[:max(1, kv_np.shape[0] // 8), :, :256])     # one chunk, an eighth of the layers
+        e1, d1, el1 = oracle_sample_step(one_np, 1)
         out["cpu_baseline"] = {
+            "single_thread_value": len(LEVELS) * 2 * el1 / d1 / 1e9,
             "value": len(LEVELS) * 2 * el / d / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{layers} of {l} layers x {cores} chunks of 256 tokens, every level, encode {e:.1f} s + decode {d:.1f} s",
             "encode_gbps_bf16_in": len(LEVELS) * 2 * el / e / 1e9}
