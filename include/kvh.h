@@ -274,6 +274,13 @@ kvh_status kvh_policy_assign_tiers(const double *freq, const kvh_option *options
                                    int n_entries, const kvh_tier *tiers, int n_tiers,
                                    int32_t *tier_out, int32_t *choice_out);
 
+/* A check callers can run on their page table before a load [host arithmetic].  KVH_ERR_PAGE_OOB
+ * if an id lies outside [0, num_pages), KVH_ERR_INVALID_ARG if an id occurs twice (two chunks
+ * decoded into the same page would race); *first_bad [host, may be NULL] receives the index of the
+ * first offending entry (for a duplicate: the later of the two). */
+kvh_status kvh_check_page_table(const int32_t *page_table, int64_t len, int32_t num_pages,
+                                int64_t *first_bad);
+
 /* ---- a load entry point that allocates nothing -------------------------------------------------
  *
  * The paper has no counterpart to this call; it exists for how the library gets deployed.  Some

@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.kvh_policy_assign.argtypes = [vp, vp, vp, i32, vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_double)]
         L.kvh_policy_assign_tiers.restype = i32
         L.kvh_policy_assign_tiers.argtypes = [vp, vp, vp, i32, vp, i32, vp, vp]
+        L.kvh_check_page_table.restype = i32
+        L.kvh_check_page_table.argtypes = [vp, i64, ctypes.c_int32, ctypes.POINTER(i64)]
         L.kvh_load_host_static.restype = i32
         L.kvh_load_host_static.argtypes = [vp, vp, vp, i32, vp, i64, ctypes.POINTER(_PoolStruct), vp, vp, u64, vp, vp]
         _lib = L
@@ -369,3 +371,12 @@ def policy_assign_tiers(freq, options, option_begin, tiers):
     _check(lib().kvh_policy_assign_tiers(f.ctypes.data, o.ctypes.data, b.ctypes.data, f.size, t.ctypes.data, len(t),
                                          tier_out.ctypes.data, choice.ctypes.data), "kvh_policy_assign_tiers")
     return tier_out, choice
+
+
+def check_page_table(page_table, num_pages: int) -> tuple[int, int]:
+    """(status, index of the first offending entry or -1) of a host page table: 0 fine, 6 an id
+    outside the pool, 1 an id used twice."""
+    t = np.ascontiguousarray(page_table, dtype=np.int32)
+    bad = ctypes.c_int64(-1)
+    st = lib().kvh_check_page_table(t.ctypes.data, t.size, num_pages, ctypes.byref(bad))
+    return st, bad.value

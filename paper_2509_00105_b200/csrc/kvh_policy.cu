@@ -142,3 +142,30 @@ extern "C" kvh_status kvh_policy_assign_tiers(const double *freq, const kvh_opti
     }
     return KVH_OK;
 }
+
+// ---- a debugging aid for callers of the decode entry points -----------------------------------
+
+// Two tokens mapped to the same page slot would make a load depend on the order in which tiles
+// happen to run.  The kernels cannot see that; the caller can check its table on the host.
+extern "C" kvh_status kvh_check_page_table(const int32_t *page_table, int64_t len, int32_t num_pages,
+                                           int64_t *first_bad)
+{
+    if (!page_table || len < 0 || num_pages <= 0) return KVH_ERR_INVALID_ARG;
+    std::vector<std::pair<int32_t, int64_t>> ids((size_t)len);
+    for (int64_t i = 0; i < len; ++i) {
+        if (page_table[i] < 0 || page_table[i] >= num_pages) {
+            if (first_bad) *first_bad = i;
+            return KVH_ERR_PAGE_OOB;
+        }
+        ids[(size_t)i] = {page_table[i], i};
+    }
+    std::sort(ids.begin(), ids.end());
+    int64_t bad = -1;
+    for (size_t i = 1; i < ids.size(); ++i)
+        if (ids[i].first == ids[i - 1].first && (bad < 0 || ids[i].second < bad)) bad = ids[i].second;
+    if (bad >= 0) {
+        if (first_bad) *first_bad = bad;
+        return KVH_ERR_INVALID_ARG;
+    }
+    return KVH_OK;
+}

@@ -194,3 +194,16 @@ def test_header_is_plain_c(tmp_path):
     inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
     subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", f"-I{inc}", str(src)],
                    check=True)
+
+
+def test_page_table_check(kvh):
+    import workloads
+    t = workloads.shuffled_page_table(500, 600, seed=1).numpy()
+    assert kvh.check_page_table(t, 600) == (0, -1)
+    u = t.copy(); u[77] = 600
+    assert kvh.check_page_table(u, 600) == (6, 77)
+    u = t.copy(); u[10] = -1
+    assert kvh.check_page_table(u, 600) == (6, 10)
+    u = t.copy(); u[300] = u[12]
+    assert kvh.check_page_table(u, 600) == (1, 300)
+    assert kvh.check_page_table(np.zeros(0, dtype=np.int32), 5) == (0, -1)
