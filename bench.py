@@ -416,6 +416,9 @@ def run_ours(args, shape: workloads.Shape):
             "value": len(LEVELS) * 2 * el / d / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{layers} of {l} layers x {cores} chunks of 256 tokens, every level, encode {e:.1f} s + decode {d:.1f} s",
             "encode_gbps_bf16_in": len(LEVELS) * 2 * el / e / 1e9}
+        # the sample's rates applied to the whole step (every level of the full context): not measured
+        full = len(LEVELS) * 2.0 * l * 2 * N * c
+        out["cpu_baseline"]["extrapolated_step_s"] = round(full / (len(LEVELS) * 2 * el) * (e + d), 1)
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
