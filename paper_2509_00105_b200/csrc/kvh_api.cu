@@ -41,18 +41,20 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     const bool want_tma = !(force && strcmp(force, "direct") == 0);
     p.bw = block_width(p.c);                             // rows wider than 1024 channels go in column blocks
     p.n_blocks = p.bw > 0 ? p.c / p.bw : 1;
-    const int64_t tiles = (int64_t)grid * p.n_blocks;
+    const bool small_pages = p.page_tokens < 16;           // a thread's rows may then span several pages
+    // narrow rows: several tiles per unit (the instance for small pages keeps one)
+    p.tpu = (p.bw > 0 && p.n_blocks == 1 && !small_pages) ? tiles_per_unit(p.bw) : 1;
+    const int64_t tiles = (int64_t)grid * p.n_blocks / p.tpu;
     if (want_tma && p.bw > 0 && tiles <= 0x7fffffffLL && p.page_tokens >= 8) {    // a lane per page id of a chunk
         int dev = 0, sms = 0, per_sm = 0;
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return KVH_ERR_CUDA;
-        const uint32_t stage = tma_stage_bytes(p.bw);
+        const uint32_t stage = tma_stage_bytes(p.bw * p.tpu);
         int stages = (int)((112u * 1024u) / stage);           // two CTAs per SM when c = 1024
         stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
         const size_t dyn = (size_t)stages * stage;
         // the instance with the channel count of the Llama-3 shapes compiled in, or the general one
-        const bool small_pages = p.page_tokens < 16;       // a thread's rows may then span several pages
         auto kernel = p.c == 1024 ? (small_pages ? decode_tma_kernel<1024, true> : decode_tma_kernel<1024, false>)
                                   : (small_pages ? decode_tma_kernel<0, true> : decode_tma_kernel<0, false>);
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess ||
@@ -150,8 +152,9 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
         EncodeParams q = p;
         q.bw = bw;
         q.n_blocks = p.c / bw;
-        auto tiles = [&](int64_t chunks) -> unsigned {   // one CTA per tile and column block; 0 if too many
-            const int64_t g = (int64_t)grid_for(chunks, p.l) * q.n_blocks;
+        q.tpu = q.n_blocks == 1 ? tiles_per_unit(bw) : 1;        // narrow rows: several tiles per unit
+        auto tiles = [&](int64_t chunks) -> unsigned {   // one CTA per unit and column block; 0 if too many
+            const int64_t g = (int64_t)grid_for(chunks, p.l) * q.n_blocks / q.tpu;
             return (grid_for(chunks, p.l) == 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;
         };
         if (tiles(n_chunks) == 0) return KVH_ERR_BAD_SHAPE;

@@ -27,6 +27,7 @@ struct DecodeParams {
     int64_t layer_stride, kv_stride, page_stride;
     int32_t num_pages, page_tokens, page_shift, l, c;   // page_tokens == 1 << page_shift
     int32_t bw, n_blocks;             // TMA-fed kernel: channels per column block (c when c <= 1024), blocks per row
+    int32_t tpu;                      // TMA-fed kernel: 32-token tiles per work unit (1, 2, 4, 8; 1 unless rows are narrow)
     int32_t *status;
 };
 

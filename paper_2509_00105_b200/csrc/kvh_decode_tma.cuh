@@ -10,7 +10,10 @@
 // the kernel runs at the speed of its writes (2 of the (b+1)/8 + 2 bytes moved per element).
 //
 // A unit is a 32-token tile of a quantised plane (<= 32*c bytes of codes + 4*c bytes of metadata)
-// or one 16-token half of a raw bf16 tile (32*c bytes), so every unit fits one stage.
+// or one 16-token half of a raw bf16 tile (32*c bytes), so every unit fits one stage.  Rows of at
+// most 512 channels would leave threads idle and make units small, so there a unit takes 2, 4 or 8
+// consecutive tiles of the plane (DecodeParams::tpu; codes and metadata of consecutive tiles are
+// contiguous in the stream) and the stage grows by the same factor.
 //
 // Every wait is bounded: a wait that runs out reports KVH_ERR_TIMEOUT, raises the CTA's abort
 // flag and the CTA leaves after its copies in flight have landed.
@@ -31,8 +34,9 @@ struct UnitInfo {
     int32_t bits;        // 16, 8, 4, 2; 0 marks the end of the CTA's work
     int32_t kv;          // 0 K, 1 V
     int32_t row0;        // first token of the unit within its chunk
-    int32_t nrows;       // tokens in the unit (1..32)
+    int32_t nrows;       // tokens in the unit (1..32 * tpu)
     int32_t pg[4];       // page ids of the page holding row0 and of the next three (pages hold >= 8 tokens)
+    const int32_t *pgs;  // the same and up to 12 more, in shared memory (units of several tiles)
     uint16_t *plane;     // pool + layer*layer_stride + kv*kv_stride
     int32_t col0, cw;    // first channel and width of the unit's column block (0, c unless rows exceed 1024 channels)
 };
@@ -113,8 +117,8 @@ __device__ __forceinline__ uint4 fma_pack8(const f32x2 (&x)[4], const f32x2 (&sc
 }
 
 // Rows of a unit are dealt to threads in runs of consecutive rows: `rpt` rows per thread (a power of
-// two: 16 when c = 1024), cut into runs of at most a page, so that a run never straddles a page;
-// `cv` is the thread's 8-channel vector within the row.
+// two, at most 16: 16 when c = 1024), cut into runs of at most a page, so that a run never straddles
+// a page or a tile; `cv` is the thread's 8-channel vector within the row.
 struct RowRun {
     int cv, first, count;       // count == 0 for idle threads
     uint16_t *dst;              // first row's destination (already offset by cv), nullptr if none
@@ -132,7 +136,8 @@ __device__ __forceinline__ RowRuns row_runs(const DecodeParams &p, const UnitInf
     RowRuns rr;
     rr.rpp = kConsumerThreads / V8;                       // row groups the CTA holds, >= 2
     int rpt = 1;
-    while (rpt * rr.rpp < kTileTokens) rpt <<= 1;         // rows per thread
+    const int unit_rows = kTileTokens * (C ? 1 : p.tpu);
+    while (rpt * rr.rpp < unit_rows) rpt <<= 1;           // rows per thread
     rr.len = SMALLPG ? min(rpt, p.page_tokens) : rpt;
     rr.n = SMALLPG ? rpt / rr.len : 1;
     rr.g = threadIdx.x / V8;
@@ -151,8 +156,10 @@ __device__ __forceinline__ RowRun row_run(const DecodeParams &p, const UnitInfo 
     r.dst = nullptr;
     if (r.count > 0) {
         const int T = u.row0 + r.first;
-        const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);      // 0..3; selects keep u in registers
-        const int32_t pg = pi == 0 ? u.pg[0] : (!SMALLPG || pi == 1) ? u.pg[1] : pi == 2 ? u.pg[2] : u.pg[3];
+        const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);
+        int32_t pg;
+        if constexpr (C == 0 && !SMALLPG) pg = u.pgs[pi];                   // 0..15: a unit of up to 8 tiles
+        else pg = pi == 0 ? u.pg[0] : (!SMALLPG || pi == 1) ? u.pg[1] : pi == 2 ? u.pg[2] : u.pg[3];   // selects keep u in registers
         r.dst = page_row<C>(p, pg, u.plane, T);              // reports an out-of-range page id
         if (r.dst) r.dst += (C ? 0 : u.col0) + 8 * r.cv; else r.count = 0;
     }
@@ -184,7 +191,9 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     if (rr.g >= rr.rpp) return;
     f32x2 lo[4], sc[4];
     {
-        const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * rr.cv;
+        // the thread's rows lie in one tile of the unit: that tile's groups
+        const int sub = (C || SMALLPG) ? 0 : (rr.g * rr.len) >> 5;
+        const uint4 *m = reinterpret_cast<const uint4 *>(meta + (size_t)sub * 4 * c) + 2 * rr.cv;
         const uint4 m0 = m[0], m1 = m[1];
         const uint32_t w[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
         float l1[8], s1[8];
@@ -265,19 +274,21 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
 //        1 = grid holds one CTA per tile and running CTAs pull further tiles through cluster
 //            launch control, so faster SMs take more tiles.
 template <int C, bool SMALLPG = false>
-__global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodeParams p, const int n_chunks,
+__global__ void __launch_bounds__(kTmaThreads, 2) decode_tma_kernel(const DecodeParams p, const int n_chunks,
                                                                  const int n_stages, const int sched)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
     __shared__ UnitInfo info[kMaxStages];
+    __shared__ int32_t unit_pg[kMaxStages][16];
     __shared__ int abort_flag;
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
 
-    const uint32_t stage_bytes = tma_stage_bytes(p.bw);
-    const uint32_t meta_off = 32u * p.bw;
+    const int tpu = C ? 1 : p.tpu;                        // tiles per unit
+    const uint32_t stage_bytes = tma_stage_bytes(p.bw * tpu);
+    const uint32_t meta_off = 32u * p.bw * tpu;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -294,7 +305,8 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
 
     if (warp == kConsumerThreads / 32) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
+        const int upc = kTilesPerChunk / tpu;             // units per chunk and plane
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * upc * p.n_blocks;
         int cur_chunk = -1;
         bool valid = false;
         kvh_chunk_desc d = p.single;
@@ -321,6 +333,9 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             int32_t pg[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) pg[i] = __shfl_sync(0xffffffffu, my_pg, (pidx + i) & 31);
+            const int32_t pg_mine = __shfl_sync(0xffffffffu, my_pg, (pidx + lane) & 31);
+            if (lane < 16) unit_pg[s][lane] = pg_mine;
+            __syncwarp();                                // lane 0's arrival below publishes these too
             uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const bool strided = row_stride != 0;
             if (lane == 0) {
@@ -357,8 +372,8 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
         auto do_tile = [&](int64_t tile_id) {
             const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share page rows
             const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % kTilesPerChunk);
-            const int64_t plane_id = row_tile / kTilesPerChunk;
+            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
+            const int64_t plane_id = row_tile / upc;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = (int)((plane_id >> 1) / p.l);
@@ -379,7 +394,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             }
             if (!valid) return;
             const int t0 = tile * kTileTokens;
-            const int nt = min(kTileTokens, d.n_tok - t0);
+            const int nt = min(kTileTokens * tpu, d.n_tok - t0);
             if (nt <= 0) return;
             const uint8_t *lay = p.streams + d.stream_off + (uint64_t)layer * L.layer_bytes();
             const uint8_t *meta = lay + L.meta_off(kv);
@@ -389,8 +404,9 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
             const int col0 = cb * p.bw;
             const uint32_t gpr = (uint32_t)p.c / kGroup;         // groups per plane row
             if (d.level == 0) {
-                for (int h = 0; ok && h < nt; h += 16) {
-                    const int rows = min(16, nt - h);
+                const int half = 16 * tpu;                       // rows of raw bf16 a stage holds
+                for (int h = 0; ok && h < nt; h += half) {
+                    const int rows = min(half, nt - h);
                     const uint8_t *src = codes + 2 * ((uint64_t)(t0 + h) * p.c + col0);
                     ok = wide ? emit(16, kv, t0 + h, rows, plane, col0, src, 2u * p.bw, 2u * p.c, nullptr, 0, 0)
                               : emit(16, kv, t0 + h, rows, plane, 0, src, round16(2u * rows * p.c), 0, nullptr, 0, 0);
@@ -407,7 +423,7 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                                         msrc, 4u * (p.bw / kGroup), 4u * gpr);
                 } else {
                     const uint32_t cbytes = round16((uint32_t)nt * p.c * b / 8);
-                    const uint32_t mbytes = kv == 0 ? 4u * p.c : round16(4u * nt * gpr);
+                    const uint32_t mbytes = kv == 0 ? 4u * p.c * ((nt + kTileTokens - 1) / kTileTokens) : round16(4u * nt * gpr);
                     ok = emit(b, kv, t0, nt, plane, 0, csrc, cbytes, 0, msrc, mbytes, 0);
                 }
             }
@@ -446,8 +462,9 @@ __global__ void __launch_bounds__(kTmaThreads) decode_tma_kernel(const DecodePar
                 abort_flag = 1;
                 break;
             }
-            const UnitInfo u = info[s];
+            UnitInfo u = info[s];
             if (u.bits == 0) break;
+            u.pgs = unit_pg[s];
             const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const uint8_t *mt = st + meta_off;
             switch (u.bits * 2 + u.kv) {                      // uniform per CTA

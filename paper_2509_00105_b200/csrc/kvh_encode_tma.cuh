@@ -23,6 +23,10 @@
 // tile), other widths and token dropping (kept runs gathered into a compact sequence) through one
 // 1-D bulk copy per row issued by the producer's lanes in parallel.
 //
+// Rows of at most 512 channels: a work unit takes 2, 4 or 8 consecutive tiles of the plane
+// (EncodeParams::tpu; they are contiguous in the source), so that a unit still fills a stage and
+// every consumer thread has a column of some tile.
+//
 // Tiles are handed out dynamically through cluster launch control, as in the decode kernel.  Every
 // wait is bounded: when one runs out the CTA reports KVH_ERR_TIMEOUT, raises its abort flag,
 // waits for its copies in flight and leaves.
@@ -56,8 +60,8 @@ struct ListedChunks {
 struct EncUnit {
     int32_t bits;          // 16, 8, 4, 2; 0 marks the end of the CTA's work
     int32_t kv;            // 0 K, 1 V
-    int32_t nt;            // tokens in the tile (1..32)
-    int32_t tile;          // tile index within the chunk
+    int32_t nt;            // tokens in the unit (1..32 * tpu)
+    int32_t tile;          // index within the chunk of the unit's first tile
     int32_t last;          // the plane's last tile clears the sections' padding
     uint32_t meta_payload, meta_padded, codes_payload, codes_padded;
     uint8_t *meta;         // the plane's metadata section in the stream
@@ -256,24 +260,26 @@ __device__ __forceinline__ void enc_process_k(uint2 (&x)[kTileTokens], RowGeom g
         enc_store_row_k<BITS, false>(x[t], lo_a, lo_b, inv_a, inv_b, mask, out + (size_t)t * row_bytes);
 }
 
-// A full tile: all 32 rows of the thread's 4 channels in registers, one pass over shared memory.
+// Full tiles (nt = 32, or a multiple of 32 when a unit holds several tiles of narrow rows): a thread
+// takes 4 channels of one tile, all 32 rows of them in registers, one pass over shared memory.
 template <int BITS>
 __device__ __forceinline__ void enc_consume_k(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
-                                              int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+                                              int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int C4 = g.cw >> 2;                            // 4-channel columns per stage row, <= 256
-    const bool active = tid < C4;
-    const int cq = active ? tid : 0;
-    const uint8_t *col = st + g.stage_col(4 * cq);
+    const int sub = C4 >= kEncGroupThreads ? 0 : tid / C4;      // which of the unit's tiles
+    const bool active = sub * kTileTokens < nt;
+    const int cq = active ? tid - sub * C4 : 0;
     const uint32_t rs = g.stage_row_bytes();
+    const uint8_t *col = st + g.stage_col(4 * cq) + (active ? sub : 0) * kTileTokens * rs;
     uint2 x[kTileTokens];
 #pragma unroll
     for (int t = 0; t < kTileTokens; ++t) x[t] = *reinterpret_cast<const uint2 *>(col + t * rs);
     enc_release(empty_bar);
-    if (active) enc_process_k<BITS>(x, g, cq, tile, meta_sec, codes_sec);
+    if (active) enc_process_k<BITS>(x, g, cq, tile + sub, meta_sec, codes_sec);
 }
 
-// The last, short tile of a chunk (nt < 32 rows): rare, so two plain passes over the rows.
+// A chunk's end that is not a whole number of tiles: rare, so two plain passes over the rows.
 // row(t) returns row t of the thread's 4 channels (column cq) as two packed bf16 pairs.
 template <int BITS, typename RowFn>
 __device__ __forceinline__ void enc_k_short(RowFn row, RowGeom g, int cq, int nt, int tile,
@@ -306,11 +312,14 @@ __device__ __noinline__ void enc_consume_k_short(const uint8_t *st, RowGeom g, i
                                                  int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int C4 = g.cw >> 2;
-    if (tid < C4) {
-        const uint8_t *col = st + g.stage_col(4 * tid);
+    const int sub = tid / C4;                            // which of the unit's tiles
+    const int nt_sub = min(kTileTokens, nt - sub * kTileTokens);
+    if (nt_sub > 0) {
+        const int cq = tid - sub * C4;
         const uint32_t rs = g.stage_row_bytes();
-        enc_k_short<BITS>([&](int t) { return *reinterpret_cast<const uint2 *>(col + t * rs); }, g, tid, nt, tile,
-                          meta_sec, codes_sec);
+        const uint8_t *col = st + g.stage_col(4 * cq) + sub * kTileTokens * rs;
+        enc_k_short<BITS>([&](int t) { return *reinterpret_cast<const uint2 *>(col + t * rs); }, g, cq, nt_sub,
+                          tile + sub, meta_sec, codes_sec);
     }
     enc_release(empty_bar);
 }
@@ -452,7 +461,7 @@ __device__ __forceinline__ void enc_consume_level(const EncUnit &u, const uint8_
     } else {
         constexpr int BITS = 16 >> LEVEL;
         if (u.kv) enc_consume_v<BITS>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
-        else if (u.nt == kTileTokens) enc_consume_k<BITS>(st, g, tid, eb, u.tile, u.meta, u.codes);
+        else if ((u.nt & (kTileTokens - 1)) == 0) enc_consume_k<BITS>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
         else enc_consume_k_short<BITS>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
     }
 }
@@ -515,7 +524,9 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
 
     if (warp == kProducerWarp) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
+        const int tpu = (C != 0) ? 1 : p.tpu;             // tiles per unit
+        const int upc = kTilesPerChunk / tpu;             // units per chunk and plane
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * upc * p.n_blocks;
         uint32_t unit = 0;
         bool ok = true;
 
@@ -530,8 +541,8 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
         auto do_tile = [&](int64_t tile_id) {
             const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share rows
             const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % kTilesPerChunk);
-            const int64_t plane_id = row_tile / kTilesPerChunk;
+            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
+            const int64_t plane_id = row_tile / upc;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), p.chunk0);
@@ -553,7 +564,7 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                 return;
             }
             const int n = d.n_tok;
-            const int nt = min(kTileTokens, n - tile * kTileTokens);
+            const int nt = min(kTileTokens * tpu, n - tile * kTileTokens);
             if (nt <= 0) return;
             const LayerLayout L = layer_layout(d.level, p.c, n);
             uint8_t *lay = p.out + d.stream_off + (uint64_t)layer * L.layer_bytes();

@@ -49,6 +49,16 @@ inline int block_width(int c)
     return 0;
 }
 
+// Tiles of 32 tokens a work unit of the TMA-fed kernels takes when rows are bw channels wide: as
+// many (1, 2, 4 or 8, a chunk has 8) as keep a unit within 1024 channels' worth of a tile, so that
+// narrow rows still give every consumer thread work and the pipeline units of useful size.
+inline int tiles_per_unit(int bw)
+{
+    int t = 1;
+    while (t < kTilesPerChunk && 2 * t * bw <= 1024) t <<= 1;
+    return t;
+}
+
 inline kvh_status launch_status()
 {
     return cudaPeekAtLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;

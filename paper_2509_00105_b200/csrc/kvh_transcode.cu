@@ -30,7 +30,7 @@ auto pick_kernel(int lin, int lout) -> void (*)(const TranscodeParams, const int
 template <typename Chunks>
 kvh_status launch(const TranscodeParams &p, int lin, int lout, int n_chunks, cudaStream_t st, const Chunks &chunks)
 {
-    const int64_t tiles = (int64_t)grid_for(n_chunks, p.l) * p.n_blocks;
+    const int64_t tiles = (int64_t)grid_for(n_chunks, p.l) * p.n_blocks / p.tpu;     // one CTA per unit
     if (grid_for(n_chunks, p.l) == 0 || tiles > 0x7fffffffLL) return KVH_ERR_BAD_SHAPE;
     const unsigned grid = (unsigned)tiles;
     int dev = 0, sms = 0;
@@ -79,6 +79,7 @@ extern "C" kvh_status kvh_transcode(const void *in_streams, uint64_t in_bytes, c
     p.l = n_layers; p.c = n_channels;
     p.bw = block_width(n_channels);
     p.n_blocks = n_channels / p.bw;
+    p.tpu = p.n_blocks == 1 ? tiles_per_unit(p.bw) : 1;              // narrow rows: several tiles per unit
     p.status = dev_status;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (level_in >= 0 || !in_descs_host || !out_descs_host)

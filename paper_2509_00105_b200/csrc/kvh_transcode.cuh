@@ -32,6 +32,7 @@ struct TranscodeParams {
     const kvh_chunk_desc *out_descs;    // device, n_chunks
     int32_t l, c;
     int32_t bw, n_blocks;               // channels per column block (c when c <= 1024), blocks per row
+    int32_t tpu;                        // 32-token tiles per work unit (1, 2, 4, 8; 1 unless rows are narrow)
     int32_t *status;
 };
 
@@ -40,7 +41,8 @@ struct TcUnit {
     int32_t bits_in;       // 16, 8, 4, 2
 };
 
-// Offset of a unit's metadata in its stage; the codes (or raw rows) start at 0.
+// Offset of a unit's metadata in its stage; the codes (or raw rows) start at 0.  c: channels per
+// stage row times the tiles a unit holds.
 __host__ __device__ __forceinline__ uint32_t tc_meta_off(int c) { return 32u * (uint32_t)c; }
 
 // q_i * 2^pos(i) for the 4 codes of one K row of a 4-channel column: x[0] = elements 0, 1 and
@@ -94,15 +96,20 @@ __device__ __forceinline__ uint2 tc_row_k(const uint8_t *codes, const f32x2 (&lo
                       pack_bf16x2_rn(__uint_as_float(c2), __uint_as_float(d)));
 }
 
-// K: a thread owns 4 channels and walks the tile's rows (any number of them).
+// K: a thread owns 4 channels of one of the unit's tiles and walks that tile's rows (any number of
+// them).
 template <int BIN, int BOUT>
 __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
-                                             int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+                                             int nt_unit, int tile0, int tpu, uint8_t *meta_sec, uint8_t *codes_sec)
 {
     const int c = g.cw;                                  // channels per stage row
-    if (tid < (c >> 2)) {
-        const int cq = tid;
-        const uint4 w4 = *reinterpret_cast<const uint4 *>(st + tc_meta_off(c) + 16 * (size_t)cq);
+    const int C4 = c >> 2;
+    const int sub = tid / C4;                            // which of the unit's tiles
+    const int nt = min(kTileTokens, nt_unit - sub * kTileTokens);
+    if (nt > 0) {
+        const int cq = tid - sub * C4;
+        const int tile = tile0 + sub;
+        const uint4 w4 = *reinterpret_cast<const uint4 *>(st + tc_meta_off(c * tpu) + 4 * (size_t)sub * c + 16 * (size_t)cq);
         const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
         float l1[4], s1[4], lo_new[4], inv[4];
         uint32_t m[4], mask[4];
@@ -125,7 +132,7 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int t
         const f32x2 lo_a = f2_make(lo_new[0], lo_new[1]), lo_b = f2_make(lo_new[2], lo_new[3]);
         const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
         const uint32_t in_bytes = (uint32_t)c * BIN / 8;
-        const uint8_t *src = st + (size_t)cq * BIN / 2;   // 4 codes = BIN / 2 bytes
+        const uint8_t *src = st + (size_t)sub * kTileTokens * in_bytes + (size_t)cq * BIN / 2;   // 4 codes = BIN / 2 bytes
         if (all_quantised) {
 #pragma unroll 8
             for (int t = 0; t < nt; ++t)
@@ -144,10 +151,10 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int t
 // V: a thread dequantises whole groups (32 codes, one metadata word) and encodes them again.
 template <int BIN, int BOUT>
 __device__ __forceinline__ void tc_consume_v(const uint8_t *st, RowGeom geom, int tid, uint64_t *empty_bar,
-                                             int nt, int tile, uint8_t *meta_sec, uint8_t *codes_sec)
+                                             int nt, int tile, int tpu, uint8_t *meta_sec, uint8_t *codes_sec)
 {
-    const int ngroups = nt * (geom.cw >> 5);             // the tile's groups, in stage order
-    const uint32_t *meta_in = reinterpret_cast<const uint32_t *>(st + tc_meta_off(geom.cw));
+    const int ngroups = nt * (geom.cw >> 5);             // the unit's groups, in stage order
+    const uint32_t *meta_in = reinterpret_cast<const uint32_t *>(st + tc_meta_off(geom.cw * tpu));
     uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec);
     const f32x2 pre01 = f2_make(Pos<BIN>::prescale(0), Pos<BIN>::prescale(1));
     const f32x2 pre23 = f2_make(Pos<BIN>::prescale(2), Pos<BIN>::prescale(3));
@@ -174,7 +181,7 @@ __device__ __forceinline__ void tc_consume_v(const uint8_t *st, RowGeom geom, in
 
 // One unit with both levels known at compile time (LOUT > LIN).
 template <int C, int LIN, int LOUT>
-__device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_t *st, int c_rt, int tid,
+__device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_t *st, int c_rt, int tpu_rt, int tid,
                                                   uint64_t *eb)
 {
     if constexpr (LIN == 0) {
@@ -182,31 +189,33 @@ __device__ __forceinline__ void tc_consume_levels(const EncUnit &u, const uint8_
     } else {
         constexpr int BIN = 16 >> LIN, BOUT = 16 >> LOUT;
         const RowGeom g = row_geom<C>(u.cw, c_rt, u.col0);
-        if (u.kv) tc_consume_v<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
-        else tc_consume_k<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, u.meta, u.codes);
+        const int tpu = C ? 1 : tpu_rt;
+        if (u.kv) tc_consume_v<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, tpu, u.meta, u.codes);
+        else tc_consume_k<BIN, BOUT>(st, g, tid, eb, u.nt, u.tile, tpu, u.meta, u.codes);
     }
 }
 template <int C, int LIN, int LOUT>
-__device__ __noinline__ void tc_consume_levels_call(const EncUnit *u, const uint8_t *st, int c_rt, int tid,
+__device__ __noinline__ void tc_consume_levels_call(const EncUnit *u, const uint8_t *st, int c_rt, int tpu_rt, int tid,
                                                     uint64_t *eb)
 {
-    tc_consume_levels<C, LIN, LOUT>(*u, st, c_rt, tid, eb);
+    tc_consume_levels<C, LIN, LOUT>(*u, st, c_rt, tpu_rt, tid, eb);
 }
 
 // LIN, LOUT >= 0: every chunk goes from LIN to LOUT (checked by the producer); -1: any mix.
 template <int C, int LIN, int LOUT>
-__device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, int c_rt, int tid, uint64_t *eb)
+__device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, int c_rt, int tpu_rt, int tid,
+                                            uint64_t *eb)
 {
     if constexpr (LIN >= 0) {
-        tc_consume_levels<C, LIN, LOUT>(u.e, st, c_rt, tid, eb);
+        tc_consume_levels<C, LIN, LOUT>(u.e, st, c_rt, tpu_rt, tid, eb);
     } else {
         switch (u.bits_in * 16 + u.e.bits) {             // uniform per CTA
-        case 16 * 16 + 8: tc_consume_levels_call<C, 0, 1>(&u.e, st, c_rt, tid, eb); break;
-        case 16 * 16 + 4: tc_consume_levels_call<C, 0, 2>(&u.e, st, c_rt, tid, eb); break;
-        case 16 * 16 + 2: tc_consume_levels_call<C, 0, 3>(&u.e, st, c_rt, tid, eb); break;
-        case 8 * 16 + 4: tc_consume_levels_call<C, 1, 2>(&u.e, st, c_rt, tid, eb); break;
-        case 8 * 16 + 2: tc_consume_levels_call<C, 1, 3>(&u.e, st, c_rt, tid, eb); break;
-        default: tc_consume_levels_call<C, 2, 3>(&u.e, st, c_rt, tid, eb); break;
+        case 16 * 16 + 8: tc_consume_levels_call<C, 0, 1>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
+        case 16 * 16 + 4: tc_consume_levels_call<C, 0, 2>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
+        case 16 * 16 + 2: tc_consume_levels_call<C, 0, 3>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
+        case 8 * 16 + 4: tc_consume_levels_call<C, 1, 2>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
+        case 8 * 16 + 2: tc_consume_levels_call<C, 1, 3>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
+        default: tc_consume_levels_call<C, 2, 3>(&u.e, st, c_rt, tpu_rt, tid, eb); break;
         }
     }
 }
@@ -246,7 +255,9 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
 
     if (warp == kProducerWarp) {
         // ------------------------------ producer warp ------------------------------
-        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * kTilesPerChunk * p.n_blocks;
+        const int tpu = C ? 1 : p.tpu;                    // tiles per unit
+        const int upc = kTilesPerChunk / tpu;             // units per chunk and plane
+        const int64_t total_tiles = (int64_t)n_chunks * p.l * 2 * upc * p.n_blocks;
         uint32_t unit = 0;
         bool ok = true;
         int cur_chunk = -1;
@@ -265,8 +276,8 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         auto do_tile = [&](int64_t tile_id) {
             const int cb = (int)(tile_id % p.n_blocks);          // column block (rows wider than 1024 channels)
             const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % kTilesPerChunk);
-            const int64_t plane_id = row_tile / kTilesPerChunk;
+            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
+            const int64_t plane_id = row_tile / upc;
             const int kv = (int)(plane_id & 1);
             const int layer = (int)((plane_id >> 1) % p.l);
             const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), 0);
@@ -290,7 +301,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
             if (!valid) return;
             const int n = di.n_tok;
             const int t0 = tile * kTileTokens;
-            const int nt = min(kTileTokens, n - t0);
+            const int nt = min(kTileTokens * tpu, n - t0);
             if (nt <= 0) return;
             const uint8_t *lay_in = p.in + di.stream_off + (uint64_t)layer * Li.layer_bytes();
             uint8_t *lay_out = p.out + dout.stream_off + (uint64_t)layer * Lo.layer_bytes();
@@ -324,10 +335,12 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
                 u.e.col0 = col0; u.e.cw = p.bw;
                 if (!wide) {
                     const uint32_t cbytes = round16((uint32_t)nt * row_bytes);
-                    const uint32_t mbytes = di.level == 0 ? 0u : kv == 0 ? 4u * p.c : round16((uint32_t)nt * mrow_bytes);
+                    const uint32_t mbytes = di.level == 0 ? 0u
+                                          : kv == 0     ? 4u * p.c * ((nt + kTileTokens - 1) / kTileTokens)
+                                                        : round16((uint32_t)nt * mrow_bytes);
                     mbar_arrive_expect_tx(&full_bar[s], cbytes + mbytes);
                     bulk_load(st, csrc, cbytes, &full_bar[s]);
-                    if (mbytes) bulk_load(st + tc_meta_off(p.bw), msrc, mbytes, &full_bar[s]);
+                    if (mbytes) bulk_load(st + tc_meta_off(p.bw * tpu), msrc, mbytes, &full_bar[s]);
                 } else {
                     const uint32_t mbytes = di.level == 0 ? 0u : kv == 0 ? 4u * p.bw : (uint32_t)nt * mrow_bytes;
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)nt * row_bytes + mbytes);
@@ -393,7 +406,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
                 if (u.e.codes_payload + tid < u.e.codes_padded) u.e.codes[u.e.codes_payload + tid] = 0;
                 if (u.e.meta_payload + tid < u.e.meta_padded) u.e.meta[u.e.meta_payload + tid] = 0;
             }
-            tc_dispatch<C, LIN, LOUT>(u, st, p.c, tid, &empty_bar[s]);
+            tc_dispatch<C, LIN, LOUT>(u, st, p.c, p.tpu, tid, &empty_bar[s]);
         }
     }
 }

@@ -84,6 +84,10 @@ SHAPES = [
     (1, 32, 1), (1, 32, 15), (2, 32, 16), (1, 64, 17), (1, 96, 31), (1, 128, 32), (2, 160, 33),
     (1, 256, 255), (1, 32, 256), (2, 64, 257), (1, 1024, 300), (1, 2048, 40), (1, 4096, 33), (3, 512, 700),
     (1, 1152, 70), (1, 1280, 33), (2, 3072, 290), (1, 2080, 35),     # wider than 1024: column blocks of 384, 640, 1024; none
+    # rows of at most 512 channels: a work unit takes 2, 4 or 8 tiles; lengths that end a unit after a
+    # whole tile, inside its second tile, and that leave whole units empty
+    (2, 512, 320), (1, 512, 256 + 33), (1, 384, 200), (1, 256, 2 * 256 + 96), (1, 256, 129), (1, 128, 130),
+    (2, 96, 300), (1, 544, 100), (1, 64, 256 + 224),
 ]
 
 
@@ -261,7 +265,7 @@ def test_bad_descriptors_are_skipped_and_reported(kvh):
 
 
 @pytest.mark.parametrize("path", ["default", "direct"])
-@pytest.mark.parametrize("l,c,N", [(1, 64, 100), (2, 1024, 300), (1, 2048, 77)])
+@pytest.mark.parametrize("l,c,N", [(1, 64, 100), (2, 1024, 300), (1, 2048, 77), (2, 512, 600), (1, 128, 333)])
 def test_page_size_other_than_16(kvh, monkeypatch, l, c, N, path):
     """Pages of 8 tokens and more go through the persistent kernel (a thread's run of rows is cut at
     page boundaries: a 32-token tile then spans up to 4 pages); smaller pages take the direct one."""
@@ -322,7 +326,7 @@ def lattice_kv(l, N, c, seed):
     return (bits >> 16).astype(np.uint16)
 
 
-@pytest.mark.parametrize("l,c,N", [(2, 1024, 512), (1, 64, 300), (1, 2048, 64)])
+@pytest.mark.parametrize("l,c,N", [(2, 1024, 512), (1, 64, 300), (1, 2048, 64), (1, 256, 300)])
 @pytest.mark.parametrize("level", [1, 2, 3])
 def test_encode_rounds_ties_like_the_oracle(kvh, l, c, N, level):
     kv_np = lattice_kv(l, N, c, seed=level * 100 + c)

@@ -23,6 +23,8 @@ CASES = [
     (1, 2048, 300, [(0, 4), (100, 60)], 2),              # rows wider than a stage: column blocks of 1024
     (1, 1152, 200, [(3, 30), (150, 41)], [1]),           # ... of 384
     (1, 3072, 90, [(0, 90)], 0),
+    (2, 512, 1500, [(0, 4), (700, 350), (1100, 90)], [3, 1]),        # narrow rows: seams inside units of two tiles
+    (1, 128, 3000, [(5, 100), (1000, 7), (2000, 333)], 2),           # ... of eight
 ]
 
 

@@ -49,7 +49,8 @@ def run_case(kvh, l, c, N, levels_in, levels_out, hint):
 
 
 @pytest.mark.parametrize("l,c,N", [(1, 1024, 300), (2, 256, 257), (1, 32, 33), (1, 96, 700), (2, 1024, 64),
-                                   (1, 2048, 70), (1, 1152, 40)])
+                                   (1, 2048, 70), (1, 1152, 40),
+                                   (2, 512, 320), (1, 512, 289), (1, 128, 256 + 130), (1, 384, 200)])   # units of 2, 8 and 2 tiles
 @pytest.mark.parametrize("pair", PAIRS)
 def test_transcode_one_pair_of_levels(kvh, l, c, N, pair):
     run_case(kvh, l, c, N, pair[0], pair[1], pair)       # the kernel specialised for the pair
