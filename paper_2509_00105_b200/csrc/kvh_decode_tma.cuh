@@ -188,7 +188,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
     const int c = C ? C : u.cw;                           // row width in the stage
     const int dstride = C ? C : p.c;                      // row width of a page
     const RowRuns rr = row_runs<C, SMALLPG>(p, u);
-    if (rr.g >= rr.rpp) return;
+    if (rr.g >= rr.rpp || rr.g * rr.len >= u.nrows) return;     // no rows: no metadata of a tile to read either
     f32x2 lo[4], sc[4];
     {
         // the thread's rows lie in one tile of the unit: that tile's groups
