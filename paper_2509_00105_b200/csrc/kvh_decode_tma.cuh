@@ -274,7 +274,7 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
 //        1 = grid holds one CTA per tile and running CTAs pull further tiles through cluster
 //            launch control, so faster SMs take more tiles.
 template <int C, bool SMALLPG = false>
-__global__ void __launch_bounds__(kTmaThreads, 2) decode_tma_kernel(const DecodeParams p, const int n_chunks,
+__global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const DecodeParams p, const int n_chunks,
                                                                  const int n_stages, const int sched)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
