@@ -39,7 +39,7 @@ kvh_status launch(const TranscodeParams &p, int lin, int lout, int n_chunks, cud
         return KVH_ERR_CUDA;
     auto kernel = p.c == 1024 ? pick_kernel<1024, Chunks>(lin, lout) : pick_kernel<0, Chunks>(lin, lout);
     if (!kernel) return KVH_ERR_BAD_LEVEL;
-    const size_t dyn = (size_t)kEncStages * (lin >= 1 ? tc_stage_bytes<1>() : tc_stage_bytes<0>());
+    const size_t dyn = lin >= 1 ? (size_t)tc_stages<1>() * tc_stage_bytes<1>() : (size_t)tc_stages<0>() * tc_stage_bytes<0>();
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return KVH_ERR_CUDA;
     const char *sched_env = getenv("KVH_ENCODE_SCHED");              // static tile stride: a measurement aid

@@ -225,15 +225,19 @@ __device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, 
 // most 8 bits plus metadata (36 KiB), which leaves room for two CTAs per SM.
 template <int LIN>
 __host__ __device__ constexpr uint32_t tc_stage_bytes() { return LIN >= 1 ? 36u * 1024u : kEncStageBytes; }
+// Stages per CTA: two of them leave room for three CTAs per SM when the source is quantised.
+template <int LIN>
+__host__ __device__ constexpr int tc_stages() { return LIN >= 1 ? 2 : kEncStages; }
 
 template <int C, int LIN, int LOUT, typename Chunks>
-__global__ void __launch_bounds__(32 + kEncGroupThreads, LIN >= 1 ? 2 : 1)
+__global__ void __launch_bounds__(32 + kEncGroupThreads, LIN >= 1 ? 3 : 1)
 transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sched, const Chunks chunks)
 {
+    constexpr int kStages = tc_stages<LIN>();
     extern __shared__ __align__(128) uint8_t stage_mem[];
-    __shared__ __align__(8) uint64_t full_bar[kEncStages];
-    __shared__ __align__(8) uint64_t empty_bar[kEncStages];
-    __shared__ TcUnit info[kEncStages];
+    __shared__ __align__(8) uint64_t full_bar[kStages];
+    __shared__ __align__(8) uint64_t empty_bar[kStages];
+    __shared__ TcUnit info[kStages];
     __shared__ int abort_flag;
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
@@ -242,7 +246,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
     constexpr int kProducerWarp = kEncGroupThreads / 32;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kEncStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kEncGroupThreads / 32);
         }
@@ -266,10 +270,10 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         LayerLayout Li = layer_layout(0, p.c, 1), Lo = Li;
 
         auto acquire = [&]() -> bool {                   // wait until the unit's stage is free
-            const int s = unit % kEncStages;
-            if (unit < (uint32_t)kEncStages) return true;
+            const int s = unit % kStages;
+            if (unit < (uint32_t)kStages) return true;
             bool w = true;
-            if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / kEncStages) - 1) & 1, &abort_flag);
+            if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / kStages) - 1) & 1, &abort_flag);
             return __shfl_sync(0xffffffffu, w, 0);
         };
 
@@ -307,7 +311,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
             uint8_t *lay_out = p.out + dout.stream_off + (uint64_t)layer * Lo.layer_bytes();
             ok = acquire();
             if (!ok) return;
-            const int s = unit % kEncStages;
+            const int s = unit % kStages;
             uint8_t *st = stage_mem + (size_t)s * tc_stage_bytes<LIN>();
             const bool wide = p.n_blocks > 1;
             const int col0 = cb * p.bw;
@@ -372,8 +376,8 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         if (ok) ok = acquire();
         if (ok) {                                        // end marker
             if (lane == 0) {
-                info[unit % kEncStages].e.bits = 0;
-                mbar_arrive(&full_bar[unit % kEncStages]);
+                info[unit % kStages].e.bits = 0;
+                mbar_arrive(&full_bar[unit % kStages]);
             }
             ++unit;
         }
@@ -384,17 +388,17 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         // Leave only after every copy issued has landed (see the encode kernel).
         if (lane == 0) {
             int never = 0;
-            const uint32_t first = unit > (uint32_t)kEncStages ? unit - kEncStages : 0;
+            const uint32_t first = unit > (uint32_t)kStages ? unit - kStages : 0;
             for (uint32_t w = first; w < unit; ++w)
-                (void)mbar_wait(&full_bar[w % kEncStages], (w / kEncStages) & 1, &never);
+                (void)mbar_wait(&full_bar[w % kStages], (w / kStages) & 1, &never);
             feed.drain();
         }
     } else {
         // ------------------------------ consumer warps ------------------------------
         const int tid = threadIdx.x;
         for (uint32_t unit = 0;; ++unit) {
-            const int s = unit % kEncStages;
-            if (!mbar_wait(&full_bar[s], (unit / kEncStages) & 1, &abort_flag)) {
+            const int s = unit % kStages;
+            if (!mbar_wait(&full_bar[s], (unit / kStages) & 1, &abort_flag)) {
                 report(p.status, KVH_ERR_TIMEOUT);
                 abort_flag = 1;
                 break;
