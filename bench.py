@@ -44,9 +44,9 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one decode launch relative to its algorithmic bytes, from the ncu capture
 # summarised in profiles/decode_tma_kernel_llama3-70b.md (dram__bytes_read + dram__bytes_write
 # on a 4096-token slice of the same workload; traffic grows in proportion to the tokens).
-DRAM_TRAFFIC_RATIO = {0: 0.981, 1: 0.973, 2: 0.967, 3: 0.963}
+DRAM_TRAFFIC_RATIO = {0: 0.981, 1: 0.973, 2: 0.967, 3: 0.964}
 # the same for one encode launch (profiles/encode_tma_kernel_llama3-70b.md)
-ENCODE_DRAM_TRAFFIC_RATIO = {0: 0.980, 1: 0.978, 2: 0.986, 3: 0.992}
+ENCODE_DRAM_TRAFFIC_RATIO = {0: 0.979, 1: 0.979, 2: 0.986, 3: 0.992}
 
 
 def measured_peak() -> tuple[float, str]:
