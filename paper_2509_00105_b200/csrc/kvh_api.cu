@@ -114,6 +114,7 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
     // wider rows in blocks of 1024 channels: the instance with the boxed stage; it wants the tensor
     // map unless tokens are gathered from kept runs
     const bool boxed = p.c != 1024 && p.bw == 1024 && (p.n_runs > 0 || make_kv_map(p, &kv_map));
+    if (p.boxes && !make_kv_map(p, &kv_map)) return KVH_ERR_CUDA;
     if (p.c == 1024) {
         kernel = level == 0 ? encode_tma_kernel<1024, 0, Chunks> : level == 1 ? encode_tma_kernel<1024, 1, Chunks>
                : level == 2 ? encode_tma_kernel<1024, 2, Chunks> : level == 3 ? encode_tma_kernel<1024, 3, Chunks>
@@ -156,6 +157,16 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
         q.bw = bw;
         q.n_blocks = p.c / bw;
         q.tpu = q.n_blocks == 1 ? tiles_per_unit(bw) : 1;        // narrow rows: several tiles per unit
+        // 768, 1280, 1536 ...: neither packed by whole tiles nor blocks of 1024: blocks of 256 channels,
+        // 4 tiles per unit, fetched as 2-D boxes (token dropping gathers rows and keeps the row copies)
+        CUtensorMap probe;
+        if (p.c % kBoxChannels == 0 && p.c % 1024 != 0 && p.c != 256 && p.c != 512 && p.n_runs == 0 &&
+            make_kv_map(p, &probe)) {                    // without a tensor map the row copies remain
+            q.bw = kBoxChannels;
+            q.n_blocks = p.c / kBoxChannels;
+            q.tpu = 1024 / kBoxChannels;
+            q.boxes = 1;
+        }
         auto tiles = [&](int64_t chunks) -> unsigned {   // one CTA per unit and column block; 0 if too many
             const int64_t g = (int64_t)grid_for(chunks, p.l) * q.n_blocks / q.tpu;
             return (grid_for(chunks, p.l) == 0 || g > 0x7fffffffLL) ? 0u : (unsigned)g;

@@ -38,6 +38,7 @@ struct EncodeParams {
     int32_t level;                 // used when descs == nullptr
     int32_t bw, n_blocks;          // TMA-fed kernel: channels per column block (c when c <= 1024) and blocks per row
     int32_t tpu;                   // TMA-fed kernel: 32-token tiles per work unit (1, 2, 4, 8; 1 unless rows are narrow)
+    int32_t boxes;                 // TMA-fed kernel: 1 = column blocks of 256 channels fetched as 2-D boxes, a box per tile
     int32_t hint_level;            // >= 0: every chunk has this level (an instance holding only its code runs); -1: any
     uint64_t full_chunk_bytes;     // kvh_level_bytes(level, l, c, 256), same case
     uint8_t *out;

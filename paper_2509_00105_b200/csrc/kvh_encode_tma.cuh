@@ -25,7 +25,10 @@
 //
 // Rows of at most 512 channels: a work unit takes 2, 4 or 8 consecutive tiles of the plane
 // (EncodeParams::tpu; they are contiguous in the source), so that a unit still fills a stage and
-// every consumer thread has a column of some tile.
+// every consumer thread has a column of some tile.  Widths that are a multiple of 256 but neither
+// one of those nor a multiple of 1024 (768, 1280, 1536 ...) are cut into column blocks of 256
+// channels and a unit takes 4 consecutive tiles of one block, each fetched as one 2-D box: in the
+// stage that is the layout of a plane 256 channels wide (EncodeParams::boxes).
 //
 // Tiles are handed out dynamically through cluster launch control, as in the decode kernel.  Every
 // wait is bounded: when one runs out the CTA reports KVH_ERR_TIMEOUT, raises its abort flag,
@@ -586,7 +589,10 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
                 u.meta = lay + L.meta_off(kv);
                 u.codes = lay + L.codes_off(kv);
                 u.col0 = cb * p.bw; u.cw = p.bw;
-                mbar_arrive_expect_tx(&full_bar[s], WIDE && p.n_runs == 0 ? 4 * kBoxBytes : (uint32_t)nt * row_bytes);
+                const uint32_t n_boxes = (uint32_t)(nt + kTileTokens - 1) / kTileTokens;
+                mbar_arrive_expect_tx(&full_bar[s], WIDE && p.n_runs == 0 ? 4 * kBoxBytes
+                                                    : p.boxes            ? n_boxes * kBoxBytes
+                                                                         : (uint32_t)nt * row_bytes);
             }
             if (p.n_blocks == 1) {
                 if (lane == 0) {
@@ -612,6 +618,15 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         tensor_load_2d(st + k * kBoxBytes, &kv_map, cb * p.bw + k * kBoxChannels, row, &full_bar[s]);
+                }
+            } else if (!WIDE && p.boxes) {
+                // blocks of 256 channels: the unit's tiles, one box of 256 channels x 32 rows each, land one
+                // behind the other (rows past the unit's last token are loaded too and ignored)
+                const int boxes = (nt + kTileTokens - 1) / kTileTokens;
+                __syncwarp();                            // the expectation is posted first
+                if (lane < boxes) {
+                    const int row = (int)(((int64_t)layer * 2 + kv) * p.src_N + j0) + lane * kTileTokens;
+                    tensor_load_2d(st + lane * kBoxBytes, &kv_map, cb * p.bw, row, &full_bar[s]);
                 }
             } else {
                 // a column block of wide rows: lane r copies row r's piece (the expectation is posted first)
