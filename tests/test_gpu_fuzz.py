@@ -12,10 +12,10 @@ from test_gpu_parity import SENTINEL, kvh, new_status, oracle_pool, sentinel_poo
 
 pytestmark = pytest.mark.gpu
 
-WIDTHS = [32, 64, 96, 128, 160, 256, 384, 512, 640, 1024, 1152, 1280, 1536, 2048, 2080]
+WIDTHS = [32, 64, 96, 128, 160, 256, 384, 512, 640, 768, 1024, 1152, 1280, 1536, 2048, 2080, 2304]
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(36))
 def test_random_case(kvh, seed):
     rng = np.random.default_rng(1000 + seed)
     c = int(rng.choice(WIDTHS))
