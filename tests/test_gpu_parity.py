@@ -89,7 +89,7 @@ SHAPES = [
     (2, 512, 320), (1, 512, 256 + 33), (1, 384, 200), (1, 256, 2 * 256 + 96), (1, 256, 129), (1, 128, 130),
     (2, 96, 300), (1, 544, 100), (1, 64, 256 + 224),
     # multiples of 256 that are neither: column blocks of 256 channels, four tiles per unit (2-D boxes in the encoder)
-    (2, 768, 290), (1, 1280, 256 + 130), (1, 1536, 300), (1, 2304, 97),
+    (2, 768, 290), (1, 1280, 256 + 130), (1, 1536, 300), (1, 2304, 97), (1, 1792, 70),
 ]
 
 

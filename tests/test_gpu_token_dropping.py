@@ -25,6 +25,8 @@ CASES = [
     (1, 3072, 90, [(0, 90)], 0),
     (2, 512, 1500, [(0, 4), (700, 350), (1100, 90)], [3, 1]),        # narrow rows: seams inside units of two tiles
     (1, 128, 3000, [(5, 100), (1000, 7), (2000, 333)], 2),           # ... of eight
+    (1, 768, 500, [(0, 4), (200, 290)], [1, 3]),                     # a width the plain encoder takes in 2-D boxes: rows gathered instead
+    (1, 1280, 300, [(10, 33), (100, 100)], 2),
 ]
 
 
