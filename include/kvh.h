@@ -30,13 +30,23 @@
  *
  * Conventions.  Pointers marked [device] are CUDA device pointers, [host]
  * host pointers.  The caller owns every buffer; the library allocates no
- * device memory and keeps no state between calls.  Device work is enqueued on
+ * device memory and keeps no state between calls (the one exception is
+ * described with kvh_load_host_static).  Device work is enqueued on
  * `stream` (a cudaStream_t passed as void*, NULL = the default stream) and
  * the call returns without waiting.  Argument errors are reported by the
  * return value with nothing enqueued.  Errors only the GPU can see (a page id
  * outside the pool, a descriptor that does not fit its buffer) make the
  * kernel skip the offending chunk or page and atomicMax the status code into
  * *dev_status [device, may be NULL]; nothing traps.  No CPU fallback exists.
+ *
+ * Waits inside the kernels.  The persistent kernels feed themselves with
+ * asynchronous copies and wait for them on shared-memory barriers.  No such
+ * wait lasts longer than 2 seconds: a CTA whose wait runs out reports
+ * KVH_ERR_TIMEOUT through *dev_status, stops taking work, lets its copies in
+ * flight land and returns, so the launch ends and the context stays usable.
+ * The work that CTA had not finished is then missing from the output; treat
+ * the whole call as failed.  In a healthy process this never happens (a wait
+ * is over within microseconds).
  */
 #ifndef KVH_H
 #define KVH_H
@@ -62,7 +72,7 @@ enum {
     KVH_ERR_BUFFER_TOO_SMALL = 5, /* stream or page table shorter than a descriptor needs */
     KVH_ERR_PAGE_OOB = 6,         /* page id outside [0, num_pages): device-reported */
     KVH_ERR_CUDA = 7,             /* a CUDA runtime call failed (launch error) */
-    KVH_ERR_TIMEOUT = 8           /* reserved: a bounded device wait ran out */
+    KVH_ERR_TIMEOUT = 8           /* a bounded wait inside a kernel ran out: device-reported */
 };
 
 /* The serving engine's paged KV pool: element (layer, kv, page, slot, ch) is at
@@ -92,6 +102,9 @@ typedef struct {
 
 int kvh_format_version(void);
 int kvh_num_levels(void);
+/* "default" for the library proper; the test builds of the same sources that select other
+ * kernels or another tile schedule at compile time answer with their own name. */
+const char *kvh_build_variant(void);
 const char *kvh_status_string(kvh_status s);
 
 /* Properties of a level: code bits per element, group size, 1 if lossless.
@@ -295,15 +308,30 @@ kvh_status kvh_check_page_table(const int32_t *page_table, int64_t len, int32_t 
  * Arguments and behaviour are those of kvh_load_host without dev_staging / staging_bytes.  The
  * descriptors' stream offsets index the host buffer and the fixed array alike, so the end of the
  * last chunk (its stream_off plus its size) must not exceed KVH_STATIC_STAGING_BYTES; a larger
- * request returns KVH_ERR_BUFFER_TOO_SMALL with nothing enqueued (split it into several calls
- * whose descriptors start again at offset 0).  The call itself creates no device or host memory.
+ * request returns KVH_ERR_BUFFER_TOO_SMALL with nothing enqueued.  Split such a request into
+ * several calls whose descriptors start again at offset 0.  Splitting stops at one chunk: a single
+ * 256-token chunk that is larger than the array cannot be served by this call at all.  A full
+ * chunk takes 1024, 576, 320 or 192 bytes per layer and channel at levels 0..3, so one chunk fits
+ * while n_layers * n_channels is at most 65,536 / 116,508 / 209,715 / 349,525; at 80 layers of
+ * 1024 channels a level-0 chunk (80 MiB) does not fit, the quantised levels (45, 25, 15 MiB) do.
  *
- * The first call on each device looks up the array's device address (with that device current)
- * and remembers it; make that first call outside any stream capture.  All calls on a device
- * share the one array and it keeps whatever the last call left there: nothing in it needs to
- * start at zero, because every byte a decode reads is copied in by the same call first.  Two
- * calls whose GPU work can overlap (different `stream`s, or several host threads) overwrite each
- * other's staged chunks; order them on one stream or with events. */
+ * What the call does create: no device memory and no host buffers, but one short-lived CUDA event
+ * per slice and direction of hand-over (created, recorded, waited on and destroyed inside the
+ * call, exactly as in kvh_load_host), and, like every launch, it makes the runtime load the code of
+ * the decode kernel instance it uses the first time that instance runs.
+ *
+ * Set-up.  The first call on each device looks up the array's device address (with that device
+ * current) and remembers it for the life of the process: the one piece of state this library
+ * keeps.  Make that first call, and one call for every pool geometry that will be used (channel
+ * count and page size select the kernel instance), outside any stream capture and before the
+ * engine claims the rest of the device's memory: the array is part of the library's device image,
+ * which is loaded as a whole, so if the image does not fit, every kvh call on that device fails
+ * with KVH_ERR_CUDA, not only this one.
+ *
+ * Sharing.  All calls on a device share the one array and it keeps whatever the last call left
+ * there: nothing in it needs to start at zero, because every byte a decode reads is copied in by
+ * the same call first.  Two calls whose GPU work can overlap (different `stream`s, or several
+ * host threads) overwrite each other's staged chunks; order them on one stream or with events. */
 #define KVH_STATIC_STAGING_BYTES (64u << 20)
 
 kvh_status kvh_load_host_static(const void *host_streams,

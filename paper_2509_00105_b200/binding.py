@@ -17,10 +17,7 @@ CHUNK_TOKENS = 256
 GROUP = 32
 NUM_LEVELS = 4
 
-import os
-
-# KVH_LIB names another build of the library (a measurement aid: comparing build variants)
-_LIB_PATH = Path(os.environ.get("KVH_LIB") or Path(__file__).resolve().parent / "libkvh.so")
+_LIB_PATH = Path(__file__).resolve().parent / "libkvh.so"
 _lib = None
 
 
@@ -61,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.kvh_num_levels.restype = i32
         L.kvh_status_string.restype = ctypes.c_char_p
         L.kvh_status_string.argtypes = [i32]
+        L.kvh_build_variant.restype = ctypes.c_char_p
         L.kvh_level_info.restype = i32
         L.kvh_level_info.argtypes = [i32, ip, ip, ip]
         L.kvh_level_bytes.restype = i32
@@ -114,6 +112,10 @@ def _ptr(t) -> int:
 
 def format_version() -> int:
     return lib().kvh_format_version()
+
+
+def build_variant() -> str:
+    return lib().kvh_build_variant().decode()
 
 
 def status_string(status: int) -> str:

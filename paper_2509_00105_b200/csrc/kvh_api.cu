@@ -1,14 +1,13 @@
 // Host side of the C ABI declared in include/kvh.h: argument validation, size
-// arithmetic and kernel launches.  No device memory is allocated here and no
-// state survives a call.
+// arithmetic and kernel launches.  No device memory is allocated here, and the
+// only state that survives a call is the per-device address of the fixed staging
+// array of kvh_load_host_static.
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "kvh.h"
-#include <stdlib.h>
-#include <string.h>
 
 #include "kvh_decode.cuh"
 #include "kvh_decode_tma.cuh"
@@ -35,10 +34,9 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
     p.c = pool->n_channels;
     const unsigned grid = grid_for(n_chunks, p.l);
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
-    // KVH_DECODE_PATH=direct forces the one-CTA-per-tile kernel (a measurement aid); the
-    // persistent TMA kernel needs a column block to fit a shared-memory stage and pages of at least 8 tokens.
-    const char *force = getenv("KVH_DECODE_PATH");
-    const bool want_tma = !(force && strcmp(force, "direct") == 0);
+    // the persistent TMA kernel needs a column block to fit a shared-memory stage and pages of at
+    // least 8 tokens; otherwise (and in the "direct" build) the one-CTA-per-tile kernel runs
+    const bool want_tma = !kPreferDirect;
     p.bw = block_width(p.c);                             // rows wider than 1024 channels go in column blocks
     p.n_blocks = p.bw > 0 ? p.c / p.bw : 1;
     const bool small_pages = p.page_tokens < 16;           // a thread's rows may then span several pages
@@ -64,10 +62,7 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kTmaThreads, dyn) != cudaSuccess ||
             per_sm < 1)
             return KVH_ERR_CUDA;
-        // KVH_DECODE_SCHED=static walks tiles with a fixed stride instead of pulling them through
-        // cluster launch control (a measurement aid)
-        const char *sched_env = getenv("KVH_DECODE_SCHED");
-        const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
+        const int sched = kTileSched;
         const int64_t resident = (int64_t)sms * per_sm;
         const unsigned pgrid = sched == 1 ? (unsigned)tiles : (unsigned)(tiles < resident ? tiles : resident);
         kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
@@ -130,17 +125,15 @@ kvh_status launch_encode_tma(const EncodeParams &p, int level, unsigned grid, in
     }
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return KVH_ERR_CUDA;
-    const char *sched_env = getenv("KVH_ENCODE_SCHED");
-    const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
+    const int sched = kTileSched;
     const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
     kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, n_chunks, sched, chunks, kv_map);
     return launch_status();
 }
 
 // Encode launch: the persistent TMA-fed kernel when rows are at most 1024 channels wide or divide
-// into column blocks, otherwise one CTA per tile reading global memory directly.
-// KVH_ENCODE_PATH=direct forces the latter and KVH_ENCODE_SCHED=static a fixed tile stride
-// (measurement aids).
+// into column blocks, otherwise (and in the "direct" build, token dropping apart) one CTA per tile
+// reading global memory directly.
 // descs_host (may be nullptr): the caller's host copy of p.descs, indexed like it.  With it the
 // chunks of each level go, as index lists in the kernel parameters, to the instance specialised for
 // that level; without it one instance that holds all levels takes the chunks in order.
@@ -150,9 +143,8 @@ kvh_status launch_encode(const EncodeParams &p, int64_t n_chunks, void *stream,
     const unsigned grid = grid_for(n_chunks, p.l);
     if (grid == 0) return KVH_ERR_BAD_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const char *force = getenv("KVH_ENCODE_PATH");
     const int bw = block_width(p.c);
-    if (bw > 0 && (p.n_runs > 0 || !(force && strcmp(force, "direct") == 0))) {
+    if (bw > 0 && (p.n_runs > 0 || !kPreferDirect)) {
         EncodeParams q = p;
         q.bw = bw;
         q.n_blocks = p.c / bw;
@@ -210,6 +202,7 @@ extern "C" {
 
 int kvh_format_version(void) { return KVH_FORMAT_VERSION; }
 int kvh_num_levels(void) { return kNumLevels; }
+const char *kvh_build_variant(void) { return kBuildVariant; }
 
 const char *kvh_status_string(kvh_status s)
 {

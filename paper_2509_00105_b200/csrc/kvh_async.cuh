@@ -45,7 +45,8 @@ __device__ __forceinline__ unsigned long long global_ns()
     return t;
 }
 // Wait for a phase of an mbarrier; false if the time limit ran out or the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long start = global_ns();
@@ -53,7 +54,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag || global_ns() - start > kWaitLimitNs) return false;
+        if (*abort_flag || global_ns() - start > limit_ns) return false;
     }
 }
 // 1-D bulk copy global -> this CTA's shared memory; bytes is a multiple of 16, both ends 16-byte aligned.
@@ -62,6 +63,24 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
+
+// 1-D bulk copy this CTA's shared memory -> global, tracked by the issuing thread's bulk groups;
+// bytes is a multiple of 16, both ends 16-byte aligned.  Shared memory written with ordinary stores
+// needs fence_async_smem() (by the writers, before the barrier that precedes the copy) first.
+__device__ __forceinline__ void bulk_store(void *dst, const void *src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(smem_addr(src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until all but the newest N bulk groups of this thread have finished READING shared memory
+// (their source may be overwritten); the global writes may still be in flight.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// Wait until every bulk group of this thread has completed, writes included.
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Makes this thread's ordinary writes to shared memory visible to the asynchronous proxy.
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // 2-D tiled TMA load: the box the tensor map describes, with its corner at element (x, y) of the
 // tensor, lands packed (row after row) at dst; its full size counts on the mbarrier, rows or columns

@@ -59,9 +59,30 @@ inline int tiles_per_unit(int bw)
     return t;
 }
 
+// Called right after a <<<>>> launch: takes the launch's error (if any) off the runtime's
+// per-thread slot, so that it is attributed to this launch and does not stick to later calls.
 inline kvh_status launch_status()
 {
-    return cudaPeekAtLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? KVH_OK : KVH_ERR_CUDA;
 }
+
+// Build variants.  The library proper has no run-time switch between its kernels.  Two further
+// builds of the same sources exist for the tests and for the scheduling comparison of the
+// benchmark: KVH_VARIANT_DIRECT takes the one-CTA-per-tile kernels wherever they apply (so that
+// the tests can check both kernel families on every shape), KVH_VARIANT_STATIC_STRIDE
+// walks tiles with a fixed stride instead of pulling them through cluster launch control.
+#if defined(KVH_VARIANT_DIRECT)
+constexpr bool kPreferDirect = true;
+constexpr int kTileSched = 1;
+constexpr const char *kBuildVariant = "direct";
+#elif defined(KVH_VARIANT_STATIC_STRIDE)
+constexpr bool kPreferDirect = false;
+constexpr int kTileSched = 0;
+constexpr const char *kBuildVariant = "static-stride";
+#else
+constexpr bool kPreferDirect = false;
+constexpr int kTileSched = 1;
+constexpr const char *kBuildVariant = "default";
+#endif
 
 }  // namespace kvh

@@ -1,8 +1,6 @@
 // kvh_transcode: host side (argument checks, choice of the kernel instance, launch).
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
-#include <string.h>
 
 #include "kvh.h"
 #include "kvh_host.cuh"
@@ -42,8 +40,7 @@ kvh_status launch(const TranscodeParams &p, int lin, int lout, int n_chunks, cud
     const size_t dyn = lin >= 1 ? (size_t)tc_stages<1>() * tc_stage_bytes<1>() : (size_t)tc_stages<0>() * tc_stage_bytes<0>();
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
         return KVH_ERR_CUDA;
-    const char *sched_env = getenv("KVH_ENCODE_SCHED");              // static tile stride: a measurement aid
-    const int sched = (sched_env && strcmp(sched_env, "static") == 0) ? 0 : 1;
+    const int sched = kTileSched;
     const unsigned pgrid = sched == 1 ? grid : (grid < (unsigned)sms ? grid : (unsigned)sms);
     kernel<<<pgrid, 32 + kEncGroupThreads, dyn, st>>>(p, n_chunks, sched, chunks);
     return launch_status();

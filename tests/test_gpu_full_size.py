@@ -1,7 +1,17 @@
-"""Parity at the sizes of the benchmark configurations, in the launch configuration bench.py
-times (one kvh_encode and one kvh_decode_batch launch over the whole context).  The oracle
-cannot run these sizes in full, so chunks are sampled: a sampled chunk's stream and its pages must
-equal the oracle's bit for bit; pages nobody owns must keep their sentinel."""
+"""Parity at the sizes of the five benchmark configurations, in the launch configuration bench.py
+times (one kvh_encode and one kvh_decode_batch launch over the whole context), at every level.
+
+Three kinds of evidence, because the oracle cannot run the largest sizes in full:
+  * against the oracle, bit for bit: every chunk of the 8K context, and chunks spread over the whole
+    launch (first, last, middle and one in about eight in between) of the larger ones: a sampled
+    chunk's stream and its pages must equal the oracle's;
+  * whole buffers, every byte: the complete stream and the complete pool of the library proper (the
+    persistent TMA-fed kernels, tiles handed out dynamically) must equal those of the "direct" build
+    (one CTA per tile, plain loads), two independent implementations; and a second run of the same
+    decode must reproduce the pool, since which CTA takes which tile changes from run to run;
+  * coverage: every page the table names is written in full, pages nobody owns keep their sentinel.
+"""
+import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -14,79 +24,147 @@ from test_gpu_parity import SENTINEL, kvh, to_np16  # noqa: F401
 
 pytestmark = pytest.mark.gpu
 
+CORES = len(os.sched_getaffinity(0))
+
+
+def spread(n_chunks, step):
+    """First, last, the two middle chunks and one in every `step` in between."""
+    return sorted(set([0, n_chunks - 1, n_chunks // 2 - 1, n_chunks // 2] + list(range(step // 2, n_chunks, step))))
+
 
 def check_sampled_chunks(kvh, chunk_src, N, level_of_chunk, sample, streams, descs, table, pool, spare_pages):
     """chunk_src(i): the source tokens of chunk i, [l][2][n][c] on the GPU; streams/descs: what the
     GPU encoded; pool: what it decoded into."""
     ptable = table.cpu().numpy()
 
-    def one(i):
+    def fetch(i):                                       # device reads stay on this thread
         src = to_np16(chunk_src(i))
         l, _, n, c = src.shape
-        assert n == min(256, N - 256 * i)
         level = level_of_chunk(i)
-        want = oracle.encode_chunk(np.ascontiguousarray(src), 0, n, level)
         off = int(descs["stream_off"][i])
-        got = streams[off:off + want.size].cpu().numpy()
+        size = oracle.level_bytes(level, l, c, n)
+        got = streams[off:off + size].cpu().numpy()
+        npg = -(-n // 16)
+        pages = torch.from_numpy(ptable[int(descs["pt_off"][i]):int(descs["pt_off"][i]) + npg].astype(np.int64))
+        have = to_np16(pool.tensor[:, :, pages.to(pool.tensor.device)])
+        return i, src, level, got, have
+
+    def one(args):                                      # the oracle's part: ctypes releases the GIL
+        i, src, level, got, have = args
+        l, _, n, c = src.shape
+        assert n == min(256, N - 256 * i)
+        want = oracle.encode_chunk(np.ascontiguousarray(src), 0, n, level)
         assert np.array_equal(got, want), f"stream of chunk {i} at level {level}"
         npg = -(-n // 16)
         ids = np.arange(npg, dtype=np.int32)
         ref = np.full(l * 2 * npg * 16 * c, SENTINEL, dtype=np.uint16)
         oracle.decode_chunk(want, level, l, c, n, ids, ref, 2 * npg * 16 * c, npg * 16 * c, 16 * c, npg)
-        ref = ref.reshape(l, 2, npg, 16, c)
-        pages = torch.from_numpy(ptable[int(descs["pt_off"][i]):int(descs["pt_off"][i]) + npg].astype(np.int64))
-        have = to_np16(pool.tensor[:, :, pages.to(pool.tensor.device)])
-        assert np.array_equal(have, ref), f"pages of chunk {i} at level {level}"
+        assert np.array_equal(have, ref.reshape(l, 2, npg, 16, c)), f"pages of chunk {i} at level {level}"
 
-    with ThreadPoolExecutor(8) as ex:
-        list(ex.map(one, sample))
+    with ThreadPoolExecutor(CORES) as ex:
+        futures = [ex.submit(one, fetch(i)) for i in sample]
+        for f in futures:
+            f.result()
     if spare_pages is not None and len(spare_pages):
         spare = to_np16(pool.tensor[:, :, torch.as_tensor(spare_pages, device=pool.tensor.device)])
         assert np.all(spare == SENTINEL)
 
 
+def assert_every_owned_row_written(pool, table):
+    """No sentinel is left in any page the table names (the contexts checked this way end on a page
+    boundary).  Layer by layer, to bound the temporary."""
+    idx = table.long()
+    sentinel = SENTINEL                                  # 0x7FC1 is positive as a signed 16-bit value
+    for layer in range(pool.tensor.shape[0]):
+        pages = pool.tensor[layer][:, idx].view(torch.int16)
+        assert not bool((pages == sentinel).any()), f"unwritten row in layer {layer}"
+
+
 def run_context(kvh, shape, seed, levels, sample):
+    direct = kvh.variant("direct")
     l, c, N = shape.n_layers, shape.n_channels, shape.n_tokens
+    assert N % 16 == 0
     kv = workloads.make_kv(l, N, c, seed=seed, device="cuda")
     n_pages = workloads.n_pages(N)
     num_pages = n_pages + 64
     perm = workloads.shuffled_page_table(num_pages, num_pages, seed=seed)
     table = perm[:n_pages].cuda()
     pool = kvh.Pool.allocate(l, num_pages, c)
+    pool_b = direct.Pool.allocate(l, num_pages, c)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     for level in levels:
         pool.tensor.view(torch.int16).fill_(SENTINEL)
+        pool_b.tensor.view(torch.int16).fill_(SENTINEL)
         descs, total = kvh.plan_chunks(l, c, N, level)
+        descs_dev = kvh.descs_to_tensor(descs, "cuda")
         streams, used = kvh.encode(kv, level, dev_status=status)
         assert used == total
-        kvh.decode_batch(streams, kvh.descs_to_tensor(descs, "cuda"), len(descs), table, pool, status)
+        kvh.decode_batch(streams, descs_dev, len(descs), table, pool, status)
         assert status.item() == 0
+        # the oracle on the sampled chunks
         check_sampled_chunks(kvh, lambda i: kv[:, :, 256 * i:min(N, 256 * i + 256)], N, lambda i: level, sample, streams,
                              descs, table, pool, perm[n_pages:].tolist())
-        del streams
+        assert_every_owned_row_written(pool, table)
+        # the other kernel family on every byte
+        streams_b, _ = direct.encode(kv, level, dev_status=status)
+        assert torch.equal(streams, streams_b), f"TMA-fed and direct encoders differ at level {level}"
+        del streams_b
+        direct.decode_batch(streams, descs_dev, len(descs), table, pool_b, status)
+        assert status.item() == 0
+        assert torch.equal(pool.tensor.view(torch.int16), pool_b.tensor.view(torch.int16)), \
+            f"TMA-fed and direct decoders differ at level {level}"
+        # the same launch again: the dynamic hand-out of tiles must not change a byte
+        pool.tensor.view(torch.int16).fill_(SENTINEL)
+        kvh.decode_batch(streams, descs_dev, len(descs), table, pool, status)
+        streams_again, _ = kvh.encode(kv, level, dev_status=status)
+        assert status.item() == 0
+        assert torch.equal(pool.tensor.view(torch.int16), pool_b.tensor.view(torch.int16))
+        assert torch.equal(streams, streams_again)
+        del streams, streams_again
 
 
-def test_llama8b_8k_every_level(kvh):
+def test_tiny_single_context_every_level(kvh):
+    s = workloads.TINY
+    run_context(kvh, s, seed=0, levels=(0, 1, 2, 3), sample=[0])
+
+
+def test_llama8b_8k_every_level_every_chunk(kvh):
     s = workloads.LLAMA8B_8K
-    run_context(kvh, s, seed=2000, levels=(0, 1, 2, 3), sample=[0, 13, 31])
+    run_context(kvh, s, seed=2000, levels=(0, 1, 2, 3), sample=list(range(workloads.n_chunks(s.n_tokens))))
 
 
 def test_llama70b_32k_every_level(kvh):
-    """The benchmark workload itself."""
+    """The benchmark workload itself: 17 of its 128 chunks against the oracle, all of it against the
+    other kernel family."""
     s = workloads.LLAMA70B_32K
-    run_context(kvh, s, seed=4000, levels=(0, 1, 2, 3), sample=[0, 127])
+    run_context(kvh, s, seed=4000, levels=(0, 1, 2, 3), sample=spread(workloads.n_chunks(s.n_tokens), 8))
 
 
 def test_llama8b_128k_offsets_beyond_32_bits(kvh):
-    """8.6e9 elements: element and byte offsets exceed 2^32 in the input, the stream and the pool."""
+    """8.6e9 elements: element and byte offsets exceed 2^32 in the input, the stream and the pool, at
+    every level."""
     s = workloads.LLAMA8B_128K
-    run_context(kvh, s, seed=5000, levels=(0, 3), sample=[0, 300, 511])
+    run_context(kvh, s, seed=5000, levels=(0, 1, 2, 3), sample=spread(workloads.n_chunks(s.n_tokens), 32))
 
 
 def test_wide_rows_llama2_7b_shape(kvh):
     """32 KV heads x 128 = 4096 channels: the TMA-fed kernels work in column blocks of 1024."""
     s = workloads.LLAMA2_7B_4K
-    run_context(kvh, s, seed=7000, levels=(0, 1, 2, 3), sample=[0, 15])
+    run_context(kvh, s, seed=7000, levels=(0, 1, 2, 3), sample=[0, 7, 15])
+
+
+def plane_checksums(pool):
+    """Two position-dependent 64-bit sums per (layer, K|V) plane (wrap-around arithmetic)."""
+    out = []
+    w = None
+    for layer in range(pool.tensor.shape[0]):
+        for kv in range(2):
+            v = pool.tensor[layer, kv].reshape(-1).view(torch.int32).to(torch.int64)
+            if w is None:
+                w = (torch.arange(v.numel(), device=v.device, dtype=torch.int64) % 65521) + 1
+            out.append((int(v.sum()), int((v * w).sum())))
+            del v
+    return out
 
 
 def test_batched_mixed_level_load_at_scale(kvh):
@@ -94,7 +172,9 @@ def test_batched_mixed_level_load_at_scale(kvh):
     lengths log-uniform in [2K, 32K] with partial last chunks, a random level per chunk, one shared
     pool (~93 GB) behind one shuffled page table, ONE decode launch over ~2,800 chunks (~48 GB of
     streams).  On a GPU with less free memory the layer count is reduced to what fits; the launch
-    geometry per layer stays the benchmark's."""
+    geometry per layer stays the benchmark's.  Two pools of this size do not fit side by side, so
+    the other kernel family and the repeated launch are compared through per-plane checksums."""
+    direct = kvh.variant("direct")
     c = 1024
     lengths = workloads.context_lengths(workloads.BATCH_N_CONTEXTS, workloads.BATCH_MIN_TOKENS,
                                         workloads.BATCH_MAX_TOKENS, seed=3000)
@@ -108,7 +188,7 @@ def test_batched_mixed_level_load_at_scale(kvh):
     per_layer = 2 * num_pages * 16 * c * 2                                   # pool
     per_layer += sum(kvh.plan_chunks(1, c, N, lv)[1] for N, lv in zip(lengths, all_levels))   # streams
     per_layer += 2 * 2 * max(lengths) * c * 2                                # one context's KV and slack
-    l = int(max(1, min(32, (free - (12 << 30)) // per_layer)))
+    l = int(max(1, min(32, (free - (16 << 30)) // per_layer)))
     if torch.cuda.get_device_properties(0).total_memory > (170 << 30):
         assert l == 32                                  # a 180 GB part runs the workload at its full size
     perm = workloads.shuffled_page_table(num_pages, num_pages, seed=3001)
@@ -117,6 +197,7 @@ def test_batched_mixed_level_load_at_scale(kvh):
     pool.tensor.view(torch.int16).fill_(SENTINEL)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
 
+    sampled_contexts = (0, 9, 17, 31, 45, 63)
     plans, total_bytes, pt_base = [], 0, 0
     for i, N in enumerate(lengths):
         descs, size = kvh.plan_chunks(l, c, N, all_levels[i], stream_base=total_bytes, pt_base=pt_base)
@@ -132,16 +213,28 @@ def test_batched_mixed_level_load_at_scale(kvh):
         local["stream_off"] -= base
         size = int(local["stream_off"][-1]) + kvh.level_bytes(int(local["level"][-1]), l, c, int(local["n_tok"][-1]))
         kvh.encode_chunks(kv, kvh.descs_to_tensor(local, "cuda"), len(local), blob[base:base + size], status)
-        if i in (0, 17, 63):
+        if i in sampled_contexts:
             last = len(levels) - 1
-            for j in (0, last // 2, last):
+            for j in sorted({0, last // 3, 2 * last // 3, last}):
                 kept[(i, j)] = kv[:, :, 256 * j:min(N, 256 * j + 256)].clone()
         del kv
     all_descs = np.concatenate([d for _, _, d in plans])
-    kvh.decode_batch(blob, kvh.descs_to_tensor(all_descs, "cuda"), len(all_descs), table, pool, status)
+    all_descs_dev = kvh.descs_to_tensor(all_descs, "cuda")
+    kvh.decode_batch(blob, all_descs_dev, len(all_descs), table, pool, status)
     assert status.item() == 0
-    for i in (0, 17, 63):
+    assert {lv for _, levels, _ in plans for lv in levels} == {0, 1, 2, 3}
+    for i in sampled_contexts:
         N, levels, descs = plans[i]
         sample = sorted(j for (ci, j) in kept if ci == i)
         check_sampled_chunks(kvh, lambda j: kept[(i, j)], N, lambda j: levels[j], sample, blob, descs, table, pool,
                              perm[total_pages:].tolist() if i == 0 else None)
+    kept.clear()
+    sums = plane_checksums(pool)
+    # the same launch again, then the other kernel family: every plane of the pool must come out the same
+    pool.tensor.view(torch.int16).fill_(SENTINEL)
+    kvh.decode_batch(blob, all_descs_dev, len(all_descs), table, pool, status)
+    assert plane_checksums(pool) == sums
+    pool.tensor.view(torch.int16).fill_(SENTINEL)
+    direct.decode_batch(blob, all_descs_dev, len(all_descs), table, direct.Pool(pool.tensor), status)
+    assert status.item() == 0
+    assert plane_checksums(pool) == sums

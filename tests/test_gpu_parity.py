@@ -19,7 +19,7 @@ def kvh():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2509_00105_b200 import _build
-    _build.build()
+    _build.build_all()
     import paper_2509_00105_b200 as k
     k.lib()
     return k
@@ -96,14 +96,12 @@ SHAPES = [
 @pytest.mark.parametrize("path", ["default", "direct"])
 @pytest.mark.parametrize("l,c,N", SHAPES)
 @pytest.mark.parametrize("level", [0, 1, 2, 3])
-def test_encode_and_decode_match_oracle(kvh, monkeypatch, l, c, N, level, path):
-    # "default" takes the persistent TMA-fed encode and decode kernels where they apply
-    # (c <= 1024); "direct" forces the one-CTA-per-tile kernels on every shape
-    for var in ("KVH_DECODE_PATH", "KVH_ENCODE_PATH"):
-        if path == "direct":
-            monkeypatch.setenv(var, "direct")
-        else:
-            monkeypatch.delenv(var, raising=False)
+def test_encode_and_decode_match_oracle(kvh, l, c, N, level, path):
+    # "default" is the library proper: the persistent TMA-fed encode and decode kernels where they
+    # apply; "direct" is the build of the same sources that takes the one-CTA-per-tile kernels on
+    # every shape
+    kvh = kvh.variant(path)
+    assert kvh.build_variant() == path
     kv = workloads.make_kv(l, N, c, seed=1000 * level + N + c, device="cuda")
     kv_np = to_np16(kv).copy()
     special_values(kv_np, N)
@@ -268,13 +266,10 @@ def test_bad_descriptors_are_skipped_and_reported(kvh):
 
 @pytest.mark.parametrize("path", ["default", "direct"])
 @pytest.mark.parametrize("l,c,N", [(1, 64, 100), (2, 1024, 300), (1, 2048, 77), (2, 512, 600), (1, 128, 333)])
-def test_page_size_other_than_16(kvh, monkeypatch, l, c, N, path):
+def test_page_size_other_than_16(kvh, l, c, N, path):
     """Pages of 8 tokens and more go through the persistent kernel (a thread's run of rows is cut at
     page boundaries: a 32-token tile then spans up to 4 pages); smaller pages take the direct one."""
-    if path == "direct":
-        monkeypatch.setenv("KVH_DECODE_PATH", "direct")
-    else:
-        monkeypatch.delenv("KVH_DECODE_PATH", raising=False)
+    kvh = kvh.variant(path)
     kv = workloads.make_kv(l, N, c, seed=12, device="cuda")
     for page_tokens in (4, 8, 32, 64, 256):
         for level in (0, 1, 3):

@@ -36,6 +36,36 @@ def test_library_exports_every_declared_symbol(kvh):
         assert hasattr(L, n), n
 
 
+def test_no_environment_variable_steers_the_library():
+    """Which kernel runs and how tiles are scheduled is fixed when the library is built: nothing in
+    the package reads the process environment."""
+    pkg = os.path.join(ROOT, "paper_2509_00105_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")) and f != "_build.py":      # the build script reads NVCC
+                text = open(os.path.join(dirpath, f)).read()
+                assert "getenv" not in text and "os.environ" not in text, f
+
+
+def test_build_variants_export_the_same_abi(kvh):
+    """The "direct" and "static" builds (other kernels / another tile schedule, chosen at compile
+    time) export every declared symbol too and say which build they are; the self-test library
+    loads and exports its one entry point."""
+    from paper_2509_00105_b200 import _build
+    libs = _build.build_all()
+    assert kvh.build_variant() == "default"
+    for name, want in (("direct", "direct"), ("static", "static-stride")):
+        v = kvh.variant(name)
+        assert v.build_variant() == want and v is kvh.variant(name)
+        L = ctypes.CDLL(str(libs[name]))
+        for n in declared_symbols():
+            assert hasattr(L, n), (name, n)
+    assert kvh.variant("default") is kvh.binding
+    with pytest.raises(ValueError):
+        kvh.variant("nonesuch")
+    assert hasattr(ctypes.CDLL(str(libs["selftest"])), "kvh_selftest_bounded_wait")
+
+
 def test_versions_and_level_info(kvh):
     assert kvh.format_version() == 1
     assert kvh.lib().kvh_num_levels() == 4
