@@ -57,6 +57,36 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (*abort_flag || global_ns() - start > limit_ns) return false;
     }
 }
+// The consumer side of a stage hand-over for a group of n_threads threads (whole warps) that take
+// every unit together.  Polling an mbarrier costs issue slots for as long as the data is not
+// there, and in a kernel that runs at the speed of memory it usually is not there yet: eight
+// polling warps spent a quarter of all issued instructions that way.  So only the group's first
+// warp polls; the others sleep on a hardware named barrier (bar_id, 1..15), which costs nothing
+// while they wait.  The first warp publishes the outcome in verdict[unit & 1] (shared memory)
+// before the barrier and every thread takes it from there, so the whole group always agrees on
+// whether to go on: a named barrier that some warps have left for good would never open again.
+// (Two slots: a warp can be at most one unit behind the first warp, the barrier sees to that.)
+// After the barrier every thread tests the mbarrier once itself; the phase is complete and cannot
+// be re-armed before this group has released the stage, so the test succeeds at once and serves
+// as the thread's own acquire of the bytes the copy wrote.
+// False if the wait ran out or the CTA is aborting; the abort flag is raised then.
+__device__ __forceinline__ bool group_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                           volatile int *verdict, uint32_t unit, int bar_id, int n_threads,
+                                           bool first_warp)
+{
+    if (first_warp) {
+        const bool ok = mbar_wait(bar, parity, abort_flag);
+        if ((threadIdx.x & 31) == 0) {
+            if (!ok) *abort_flag = 1;
+            verdict[unit & 1] = ok ? 1 : 0;
+        }
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
+    const bool ok = verdict[unit & 1] != 0;
+    if (ok) (void)mbar_try_wait(bar, parity);
+    return ok;
+}
+
 // 1-D bulk copy global -> this CTA's shared memory; bytes is a multiple of 16, both ends 16-byte aligned.
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {

@@ -65,6 +65,15 @@ template <> struct Pos<8> {
     __device__ static __forceinline__ float prescale(int) { return 1.0f; }
 };
 
+// (a & mask) | c in one logic instruction (mask an immediate)
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "n"(MASK), "r"(c));
+    return d;
+}
+
 // q_i * 2^pos(i) as floats, for i = 0..7, from the 8 codes of one thread: x[k] holds elements 2k and
 // 2k+1 (the subtraction of 2^23 is exact, two elements per instruction)
 template <int BITS>
@@ -73,23 +82,20 @@ __device__ __forceinline__ void spread8(const uint8_t *src, f32x2 (&x)[4])
     constexpr uint32_t magic = 0x4b000000u;
     uint32_t m[8];
     if constexpr (BITS == 2) {
-        // (w | magic) & (field | magic) == (w & field) | magic since w has no bit in common with
-        // magic: one logic op per code with a single immediate
+        // one logic op per code: the field is masked where it stands and lands in the mantissa of 2^23
         const uint32_t w = *reinterpret_cast<const uint16_t *>(src);
-        const uint32_t wm = w | magic, tm = (w >> 8) | magic;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            m[i] = wm & ((3u << (2 * i)) | magic);
-            m[i + 4] = tm & ((3u << (2 * i)) | magic);
-        }
+        const uint32_t t = w >> 8;
+        m[0] = and_or<0x03u>(w, magic); m[1] = and_or<0x0cu>(w, magic);
+        m[2] = and_or<0x30u>(w, magic); m[3] = and_or<0xc0u>(w, magic);
+        m[4] = and_or<0x03u>(t, magic); m[5] = and_or<0x0cu>(t, magic);
+        m[6] = and_or<0x30u>(t, magic); m[7] = and_or<0xc0u>(t, magic);
     } else if constexpr (BITS == 4) {
         const uint32_t w = *reinterpret_cast<const uint32_t *>(src);
-        const uint32_t wm = (w & 0xffffu) | magic, tm = (w >> 16) | magic;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            m[i] = wm & ((15u << (4 * i)) | magic);
-            m[i + 4] = tm & ((15u << (4 * i)) | magic);
-        }
+        const uint32_t t = w >> 16;
+        m[0] = and_or<0x000fu>(w, magic); m[1] = and_or<0x00f0u>(w, magic);
+        m[2] = and_or<0x0f00u>(w, magic); m[3] = and_or<0xf000u>(w, magic);
+        m[4] = and_or<0x000fu>(t, magic); m[5] = and_or<0x00f0u>(t, magic);
+        m[6] = and_or<0x0f00u>(t, magic); m[7] = and_or<0xf000u>(t, magic);
     } else {
         const uint2 w = *reinterpret_cast<const uint2 *>(src);
 #pragma unroll
@@ -200,7 +206,7 @@ __device__ __forceinline__ void consume_k(const DecodeParams &p, const UnitInfo 
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             decode_params<BITS>(w[i], l1[i], s1[i]);
-            s1[i] = __fmul_rn(s1[i], Pos<BITS>::prescale(i));
+            if constexpr (BITS != 8) s1[i] = __fmul_rn(s1[i], Pos<BITS>::prescale(i));
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -256,7 +262,8 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
                     const float s0 = __shfl_sync(quad, mine, (lane & ~3) | j);
                     const float l1 = bf16_lo_to_f32(mrow[(size_t)(kb + j) * groups]);
                     const f32x2 ss = f2_make(s0, s0);
-                    const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);      // exact: powers of two
+                    f32x2 sa = ss, sb = ss;                  // at 8 bits a code sits at bit 0: nothing to undo
+                    if constexpr (BITS != 8) { sa = f2_mul(ss, pre01); sb = f2_mul(ss, pre23); }   // exact: powers of two
                     const f32x2 ll = f2_make(l1, l1);
                     const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
                     f32x2 x[4];
@@ -267,6 +274,118 @@ __device__ __forceinline__ void consume_v(const DecodeParams &p, const UnitInfo 
                 }
             }
         }
+    }
+}
+
+// ---- full tiles at a compiled-in row width, pages of at least 16 tokens -----------------------
+//
+// Nearly every unit is one of these, and for them everything but the data is a constant: a thread
+// has kRows consecutive rows inside one page, so the row loop unrolls completely, every shared-memory
+// and global offset is an immediate, and no row needs a branch or an address computation.
+template <int C>
+struct FullTile {
+    static constexpr int V8 = C >> 3;                              // 16-byte vectors per row
+    static constexpr int kRowGroups = kConsumerThreads / V8;       // row groups the CTA holds
+    static constexpr int kRows = kTileTokens / kRowGroups;         // rows per thread (16 at c = 1024)
+    static_assert(C % 256 == 0 && kRows * kRowGroups == kTileTokens && kRows % 4 == 0, "row width");
+    int cv, first;
+    uint16_t *dst;                                                 // row `first`, the thread's 8 channels; nullptr: page id out of range
+    __device__ __forceinline__ FullTile(const DecodeParams &p, const UnitInfo &u)
+    {
+        const int g = threadIdx.x / V8;
+        cv = threadIdx.x - g * V8;
+        first = g * kRows;
+        const int T = u.row0 + first;
+        const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);      // 0 or 1
+        dst = page_row<C>(p, pi ? u.pg[1] : u.pg[0], u.plane, T);           // reports an out-of-range page id
+        if (dst) dst += 8 * cv;
+    }
+};
+
+template <int C>
+__device__ __forceinline__ void consume_raw_full(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes)
+{
+    // a raw unit is a 16-token half of a tile: rows [0, 16) of the stage
+    constexpr int V8 = C >> 3, kRowGroups = kConsumerThreads / V8, kRows = 16 / kRowGroups;
+    const int g = threadIdx.x / V8, cv = threadIdx.x - g * V8;
+    const int first = g * kRows, T = u.row0 + first;
+    const int pi = (T >> p.page_shift) - (u.row0 >> p.page_shift);
+    uint16_t *row = page_row<C>(p, pi ? u.pg[1] : u.pg[0], u.plane, T);
+    if (!row) return;
+    const uint4 *src = reinterpret_cast<const uint4 *>(codes) + (size_t)first * V8 + cv;
+    uint4 *dst = reinterpret_cast<uint4 *>(row) + cv;
+    uint4 v[kRows];
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) v[k] = src[k * V8];
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) dst[k * V8] = v[k];
+}
+
+template <int BITS, int C>
+__device__ __forceinline__ void consume_k_full(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
+                                               const uint8_t *meta)
+{
+    const FullTile<C> t(p, u);
+    f32x2 lo[4], sc[4];
+    {
+        const uint4 *m = reinterpret_cast<const uint4 *>(meta) + 2 * t.cv;
+        const uint4 m0 = m[0], m1 = m[1];
+        const uint32_t w[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+        float l1[8], s1[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            decode_params<BITS>(w[i], l1[i], s1[i]);
+            if constexpr (BITS != 8) s1[i] = __fmul_rn(s1[i], Pos<BITS>::prescale(i));
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            lo[k] = f2_make(l1[2 * k], l1[2 * k + 1]);
+            sc[k] = f2_make(s1[2 * k], s1[2 * k + 1]);
+        }
+    }
+    if (!t.dst) return;
+    constexpr uint32_t row_bytes = (uint32_t)C * BITS / 8;
+    const uint8_t *src = codes + (size_t)t.first * row_bytes + (size_t)t.cv * BITS;
+#pragma unroll
+    for (int k = 0; k < FullTile<C>::kRows; ++k) {
+        f32x2 x[4];
+        spread8<BITS>(src + k * row_bytes, x);
+        *reinterpret_cast<uint4 *>(t.dst + k * C) = fma_pack8(x, sc, lo);
+    }
+}
+
+template <int BITS, int C>
+__device__ __forceinline__ void consume_v_full(const DecodeParams &p, const UnitInfo &u, const uint8_t *codes,
+                                               const uint8_t *meta)
+{
+    const FullTile<C> t(p, u);
+    constexpr int kRows = FullTile<C>::kRows, groups = C / kGroup;
+    constexpr uint32_t row_bytes = (uint32_t)C * BITS / 8;
+    const int lane = threadIdx.x & 31;
+    // the 4 lanes that share every group of this thread's rows each derive the scale of every fourth
+    // row; all 32 lanes of a warp are here together (a warp's lanes share their rows and their page)
+    const uint32_t *mrow = reinterpret_cast<const uint32_t *>(meta) + (size_t)t.first * groups + (t.cv >> 2);
+    float mine[kRows / 4];
+#pragma unroll
+    for (int i = 0; i < kRows / 4; ++i) {
+        float unused;
+        decode_params<BITS>(mrow[((lane & 3) + 4 * i) * groups], unused, mine[i]);
+    }
+    const f32x2 pre01 = f2_make(Pos<BITS>::prescale(0), Pos<BITS>::prescale(1));
+    const f32x2 pre23 = f2_make(Pos<BITS>::prescale(2), Pos<BITS>::prescale(3));
+    const uint8_t *src = codes + (size_t)t.first * row_bytes + (size_t)t.cv * BITS;
+#pragma unroll
+    for (int k = 0; k < kRows; ++k) {
+        const float s0 = __shfl_sync(0xffffffffu, mine[k >> 2], (lane & ~3) | (k & 3));
+        const float l1 = bf16_lo_to_f32(mrow[k * groups]);
+        const f32x2 ss = f2_make(s0, s0), ll = f2_make(l1, l1);
+        f32x2 sa = ss, sb = ss;
+        if constexpr (BITS != 8) { sa = f2_mul(ss, pre01); sb = f2_mul(ss, pre23); }      // exact: powers of two
+        const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+        f32x2 x[4];
+        spread8<BITS>(src + k * row_bytes, x);
+        const uint4 v = fma_pack8(x, sc, lo);
+        if (t.dst) *reinterpret_cast<uint4 *>(t.dst + k * C) = v;
     }
 }
 
@@ -283,6 +402,7 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
     __shared__ UnitInfo info[kMaxStages];
     __shared__ int32_t unit_pg[kMaxStages][16];
     __shared__ int abort_flag;
+    __shared__ int wait_verdict[2];
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
 
@@ -457,9 +577,8 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
         // ------------------------------ consumer warps ------------------------------
         for (uint32_t unit = 0;; ++unit) {
             const int s = unit % n_stages;
-            if (!mbar_wait(&full_bar[s], (unit / n_stages) & 1, &abort_flag)) {
-                report(p.status, KVH_ERR_TIMEOUT);
-                abort_flag = 1;
+            if (!group_wait(&full_bar[s], (unit / n_stages) & 1, &abort_flag, wait_verdict, unit, 1, kConsumerThreads, warp == 0)) {
+                if (threadIdx.x == 0) report(p.status, KVH_ERR_TIMEOUT);
                 break;
             }
             UnitInfo u = info[s];
@@ -467,6 +586,23 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
             u.pgs = unit_pg[s];
             const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
             const uint8_t *mt = st + meta_off;
+            bool done = false;
+            if constexpr (C != 0 && !SMALLPG) {
+                // the common case by far: a whole tile (or, raw, a whole 16-token half of one)
+                if (u.nrows == (u.bits == 16 ? 16 : kTileTokens)) {
+                    switch (u.bits * 2 + u.kv) {              // uniform per CTA
+                    case 32: case 33: consume_raw_full<C>(p, u, st); break;
+                    case 16: consume_k_full<8, C>(p, u, st, mt); break;
+                    case 17: consume_v_full<8, C>(p, u, st, mt); break;
+                    case 8: consume_k_full<4, C>(p, u, st, mt); break;
+                    case 9: consume_v_full<4, C>(p, u, st, mt); break;
+                    case 4: consume_k_full<2, C>(p, u, st, mt); break;
+                    default: consume_v_full<2, C>(p, u, st, mt); break;
+                    }
+                    done = true;
+                }
+            }
+            if (!done)
             switch (u.bits * 2 + u.kv) {                      // uniform per CTA
             case 32: case 33: consume_raw<C, SMALLPG>(p, u, st); break;
             case 16: consume_k<8, C, SMALLPG>(p, u, st, mt); break;

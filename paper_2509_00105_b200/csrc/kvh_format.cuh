@@ -69,6 +69,22 @@ constexpr float kRangeMax = 3.402823466e+38f;
 __device__ __forceinline__ float bf16_lo_to_f32(uint32_t pair) { return __uint_as_float(pair << 16); }
 __device__ __forceinline__ float bf16_hi_to_f32(uint32_t pair) { return __uint_as_float(pair & 0xffff0000u); }
 
+// r / qmax for qmax = 3, 15, 255, correctly rounded, in three instructions instead of the division
+// routine.  With c = RN(1 / qmax) and q0 = RN(r c), the remainder r - qmax q0 comes out exact from
+// one fused multiply-add, and q0 + rem c, rounded once, is the correctly rounded quotient.  The
+// sequence equals IEEE division bit for bit on every binary32 r in [2^-100, FLT_MAX] for the three
+// divisors (checked exhaustively on the host: tests/test_division_by_constant.py); r outside that
+// range never gets here.
+template <int BITS>
+__device__ __forceinline__ float div_by_qmax(float r)
+{
+    constexpr float qmax = (float)((1 << BITS) - 1);
+    constexpr float c = 1.0f / qmax;
+    const float q0 = __fmul_rn(r, c);
+    const float rem = __fmaf_rn(-qmax, q0, r);
+    return __fmaf_rn(rem, c, q0);
+}
+
 // scale = (max - min) / qmax and lo = min for decode, from one metadata word
 template <int BITS>
 __device__ __forceinline__ void decode_params(uint32_t meta, float &lo, float &scale)
@@ -76,7 +92,7 @@ __device__ __forceinline__ void decode_params(uint32_t meta, float &lo, float &s
     lo = bf16_lo_to_f32(meta);
     const float r = __fsub_rn(bf16_hi_to_f32(meta), lo);
     const bool ok = (r >= kRangeMin) && (r <= kRangeMax);
-    scale = ok ? __fdiv_rn(r, (float)((1 << BITS) - 1)) : 0.0f;
+    scale = ok ? div_by_qmax<BITS>(r) : 0.0f;
 }
 
 // inv = qmax / (max - min) for encode

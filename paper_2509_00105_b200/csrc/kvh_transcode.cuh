@@ -53,13 +53,13 @@ __device__ __forceinline__ void spread4(const uint8_t *src, f32x2 (&x)[2])
     constexpr uint32_t magic = 0x4b000000u;
     uint32_t m[4];
     if constexpr (BITS == 2) {
-        const uint32_t wm = (uint32_t)*src | magic;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m[i] = wm & ((3u << (2 * i)) | magic);
+        const uint32_t w = *src;
+        m[0] = and_or<0x03u>(w, magic); m[1] = and_or<0x0cu>(w, magic);
+        m[2] = and_or<0x30u>(w, magic); m[3] = and_or<0xc0u>(w, magic);
     } else if constexpr (BITS == 4) {
-        const uint32_t wm = (uint32_t)*reinterpret_cast<const uint16_t *>(src) | magic;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m[i] = wm & ((15u << (4 * i)) | magic);
+        const uint32_t w = *reinterpret_cast<const uint16_t *>(src);
+        m[0] = and_or<0x000fu>(w, magic); m[1] = and_or<0x00f0u>(w, magic);
+        m[2] = and_or<0x0f00u>(w, magic); m[3] = and_or<0xf000u>(w, magic);
     } else {
         const uint32_t w = *reinterpret_cast<const uint32_t *>(src);
 #pragma unroll
@@ -239,6 +239,7 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
     __shared__ __align__(8) uint64_t empty_bar[kStages];
     __shared__ TcUnit info[kStages];
     __shared__ int abort_flag;
+    __shared__ int wait_verdict[2];
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
 
@@ -398,9 +399,19 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         const int tid = threadIdx.x;
         for (uint32_t unit = 0;; ++unit) {
             const int s = unit % kStages;
-            if (!mbar_wait(&full_bar[s], (unit / kStages) & 1, &abort_flag)) {
-                report(p.status, KVH_ERR_TIMEOUT);
-                abort_flag = 1;
+            // quantised sources: three CTAs per SM, so one polling warp per CTA and a named barrier for the
+            // rest (group_wait); a level-0 source is the encoder's one CTA per SM, whose warps drift apart by
+            // design and poll for themselves
+            bool ready;
+            if constexpr (LIN >= 1) {
+                ready = group_wait(&full_bar[s], (unit / kStages) & 1, &abort_flag, wait_verdict, unit, 1, kEncGroupThreads,
+                                   warp == 0);
+            } else {
+                ready = mbar_wait(&full_bar[s], (unit / kStages) & 1, &abort_flag);
+                if (!ready) abort_flag = 1;
+            }
+            if (!ready) {
+                if (LIN < 1 || tid == 0) report(p.status, KVH_ERR_TIMEOUT);
                 break;
             }
             const TcUnit u = info[s];

@@ -73,3 +73,29 @@ def test_reference_arm_runs_on_rank_zero_only():
     out = json.loads(lines[0])
     assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["cpu_baseline"]["kind"] == "oracle"
     assert out["value"] > 0 and out["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` without torchrun around it: the script starts two ranks itself (the
+    CPU arm here, so no GPU is needed); again one JSON line, from rank 0, for a job of two."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["OMP_NUM_THREADS"] = "1"
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+           "--warmup", "0", "--workload", "tiny"]
+    p = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["impl"] == "reference" and out["n_gpus"] == 2 and out["config"]["workload"] == "tiny"
+
+
+def test_every_workload_has_a_config_without_touching_a_device():
+    sys.path.insert(0, ROOT)
+    import bench
+    names = [bench.workload_config(w)["workload"] for w in bench.WORKLOAD_NAMES]
+    assert names == ["tiny", "llama3-8b-8k", "batch-64", "llama3-70b-32k", "llama3-8b-128k"]
+    batch = bench.workload_config("batch-64")
+    assert batch["n_contexts"] == 64 and 64 * 2048 <= batch["n_tokens"] <= 64 * 32768
+    assert bench.workload_config("llama3-70b-32k")["n_tokens"] == 32768
+    assert len(bench.kernel_source_digest()) == 16
