@@ -100,24 +100,29 @@ __device__ __forceinline__ RowGeom row_geom(int cw, int cf, int col0)
     else return RowGeom{cw, cf, col0, false};
 }
 
-// Both elements of a packed bf16 pair: 2^23 + code as raw float bits (see biased_code()).  With
-// MASKED the value of a channel whose group is stored flat is replaced by 0 first, so that its
-// code is 0 even when x - min overflows.
+// Both elements of a packed bf16 pair: 2^23 + code as raw float bits (adding 2^23 to
+// s = (x - min) * inv leaves rint(s), ties to even, in the low mantissa bits).  With MASKED the value
+// of a channel whose group is stored flat is replaced by 0 first, so that its code is 0 even when
+// x - min overflows.
+// The product must be rounded before 2^23 is added.  The assembler contracts a packed mul followed
+// by a packed add into one fused multiply-add even with .rn on both, which skips that rounding and
+// moves a code wherever the product rounds to a tie; it does the same to fma(s, 1.0, 2^23) once it
+// has folded the literal 1.0 away.  With a multiplier it cannot know, the fma stays: it rounds
+// s * 1 + 2^23 once, exactly like an add, and cannot absorb the mul.
+__device__ __forceinline__ void biased_pair_f32(f32x2 x, f32x2 lo2, f32x2 inv2, uint32_t &ta, uint32_t &tb)
+{
+    const f32x2 magic = f2_from_bits(0x4b000000u, 0x4b000000u);
+    const f32x2 s = f2_mul(f2_sub(x, lo2), inv2);
+    const float one = kRuntimeOne;
+    f2_bits(f2_fma(s, f2_make(one, one), magic), ta, tb);
+}
 template <bool MASKED>
 __device__ __forceinline__ void biased_pair(uint32_t w, f32x2 lo2, f32x2 inv2, uint32_t mask_a, uint32_t mask_b,
                                             uint32_t &ta, uint32_t &tb)
 {
     uint32_t a = w << 16, b = w & 0xffff0000u;
     if (MASKED) { a &= mask_a; b &= mask_b; }
-    const f32x2 magic = f2_from_bits(0x4b000000u, 0x4b000000u);
-    // The product must be rounded before 2^23 is added.  The assembler contracts a packed mul
-    // followed by a packed add into one fused multiply-add even with .rn on both, which skips that
-    // rounding and moves a code wherever the product rounds to a tie; it does the same to
-    // fma(s, 1.0, 2^23) once it has folded the literal 1.0 away.  With a multiplier it cannot know,
-    // the fma stays: it rounds s * 1 + 2^23 once, exactly like an add, and cannot absorb the mul.
-    const f32x2 s = f2_mul(f2_sub(f2_from_bits(a, b), lo2), inv2);
-    const float one = kRuntimeOne;
-    f2_bits(f2_fma(s, f2_make(one, one), magic), ta, tb);
+    biased_pair_f32(f2_from_bits(a, b), lo2, inv2, ta, tb);
 }
 
 // Four biased codes (0x4b000000 + q) into the low 4 * BITS bits.  For 2 and 4 bits the biases end
@@ -186,6 +191,13 @@ __device__ __forceinline__ void enc_consume_raw(const uint8_t *st, RowGeom g, in
 // ---- K: one group per channel -------------------------------------------------------------------
 
 // Codes of one row of a 4-channel column, stored with the width the level needs.
+template <int BITS>
+__device__ __forceinline__ void store_codes4(uint32_t packed, uint8_t *o)
+{
+    if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(o) = packed;
+    if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(o) = (uint16_t)packed;
+    if constexpr (BITS == 2) *o = (uint8_t)packed;
+}
 template <int BITS, bool MASKED>
 __device__ __forceinline__ void enc_store_row_k(uint2 x, f32x2 lo_a, f32x2 lo_b, f32x2 inv_a, f32x2 inv_b,
                                                 const uint32_t (&mask)[4], uint8_t *o)
@@ -193,10 +205,18 @@ __device__ __forceinline__ void enc_store_row_k(uint2 x, f32x2 lo_a, f32x2 lo_b,
     uint32_t t0, t1, t2, t3;
     biased_pair<MASKED>(x.x, lo_a, inv_a, mask[0], mask[1], t0, t1);
     biased_pair<MASKED>(x.y, lo_b, inv_b, mask[2], mask[3], t2, t3);
-    const uint32_t packed = pack4_low<BITS>(t0, t1, t2, t3);
-    if constexpr (BITS == 8) *reinterpret_cast<uint32_t *>(o) = packed;
-    if constexpr (BITS == 4) *reinterpret_cast<uint16_t *>(o) = (uint16_t)packed;
-    if constexpr (BITS == 2) *o = (uint8_t)packed;
+    store_codes4<BITS>(pack4_low<BITS>(t0, t1, t2, t3), o);
+}
+// The same for a row given as four binary32 values (two pairs) that are exact in bf16; a channel
+// stored flat has inv = 0 and must not hold a value whose distance from min overflows.
+template <int BITS>
+__device__ __forceinline__ void enc_store_row_k_f32(f32x2 xa, f32x2 xb, f32x2 lo_a, f32x2 lo_b, f32x2 inv_a, f32x2 inv_b,
+                                                    uint8_t *o)
+{
+    uint32_t t0, t1, t2, t3;
+    biased_pair_f32(xa, lo_a, inv_a, t0, t1);
+    biased_pair_f32(xb, lo_b, inv_b, t2, t3);
+    store_codes4<BITS>(pack4_low<BITS>(t0, t1, t2, t3), o);
 }
 
 // Metadata words (min | max << 16) of 4 channels from their packed ranges, and what follows
@@ -360,6 +380,54 @@ __device__ __forceinline__ uint32_t enc_range_v(const uint4 (&x)[4])
     return __byte_perm(mn, mx, 0x5410);
 }
 
+// Code words of one 16-byte piece (8 elements) of a group from their 8 biased codes: W words, 2 at
+// 8 bits, else 1 (at 2 bits its low 16 bits count).
+template <int BITS, int W>
+__device__ __forceinline__ void pack_piece_v(const uint32_t (&t)[8], uint32_t (&w)[W])
+{
+    const uint32_t a = pack4_low<BITS>(t[0], t[1], t[2], t[3]);
+    const uint32_t b = pack4_low<BITS>(t[4], t[5], t[6], t[7]);
+    if constexpr (BITS == 8) { w[0] = a; w[1] = b; }
+    if constexpr (BITS == 4) w[0] = __byte_perm(a, b, 0x5410);
+    if constexpr (BITS == 2) w[0] = __byte_perm(a, b, 0x0040);       // 16 bits; the upper half is dropped later
+}
+// A piece given as 4 packed bf16 pairs ...
+template <int BITS, int W>
+__device__ __forceinline__ void enc_piece_v(const uint4 &x, f32x2 lo2, f32x2 inv2, uint32_t (&w)[W])
+{
+    uint32_t t[8];
+    biased_pair<false>(x.x, lo2, inv2, 0, 0, t[0], t[1]);
+    biased_pair<false>(x.y, lo2, inv2, 0, 0, t[2], t[3]);
+    biased_pair<false>(x.z, lo2, inv2, 0, 0, t[4], t[5]);
+    biased_pair<false>(x.w, lo2, inv2, 0, 0, t[6], t[7]);
+    pack_piece_v<BITS, W>(t, w);
+}
+// ... or as 8 binary32 values (4 pairs) that are exact in bf16.
+template <int BITS, int W>
+__device__ __forceinline__ void enc_piece_v_f32(const f32x2 (&x)[4], f32x2 lo2, f32x2 inv2, uint32_t (&w)[W])
+{
+    uint32_t t[8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) biased_pair_f32(x[k], lo2, inv2, t[2 * k], t[2 * k + 1]);
+    pack_piece_v<BITS, W>(t, w);
+}
+
+// The four pieces' code words of a group, in piece order, to the stream.
+template <int BITS, int W>
+__device__ __forceinline__ void enc_store_group_v(const uint32_t (&p)[4][W], uint8_t *codes_out)
+{
+    if constexpr (BITS == 8) {
+        uint4 *o = reinterpret_cast<uint4 *>(codes_out);
+        o[0] = make_uint4(p[0][0], p[0][1], p[1][0], p[1][1]);
+        o[1] = make_uint4(p[2][0], p[2][1], p[3][0], p[3][1]);
+    }
+    if constexpr (BITS == 4)
+        *reinterpret_cast<uint4 *>(codes_out) = make_uint4(p[0][0], p[1][0], p[2][0], p[3][0]);
+    if constexpr (BITS == 2)
+        *reinterpret_cast<uint2 *>(codes_out) = make_uint2(__byte_perm(p[0][0], p[1][0], 0x5410),
+                                                           __byte_perm(p[2][0], p[3][0], 0x5410));
+}
+
 // One group with its metadata word m known: store m and the codes.  x[j] is the 16-byte piece
 // number (j + rot) & 3 of the group's 64 bytes (ROTATED), or simply piece j.
 template <int BITS, bool ROTATED = true>
@@ -374,18 +442,7 @@ __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32
     if (inv != 0.0f) {
         const f32x2 lo2 = f2_make(lo, lo), inv2 = f2_make(inv, inv);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t t[8];
-            biased_pair<false>(x[j].x, lo2, inv2, 0, 0, t[0], t[1]);
-            biased_pair<false>(x[j].y, lo2, inv2, 0, 0, t[2], t[3]);
-            biased_pair<false>(x[j].z, lo2, inv2, 0, 0, t[4], t[5]);
-            biased_pair<false>(x[j].w, lo2, inv2, 0, 0, t[6], t[7]);
-            const uint32_t a = pack4_low<BITS>(t[0], t[1], t[2], t[3]);
-            const uint32_t b = pack4_low<BITS>(t[4], t[5], t[6], t[7]);
-            if constexpr (BITS == 8) { p[j][0] = a; p[j][1] = b; }
-            if constexpr (BITS == 4) p[j][0] = __byte_perm(a, b, 0x5410);
-            if constexpr (BITS == 2) p[j][0] = __byte_perm(a, b, 0x0040);     // 16 bits; the upper half is dropped below
-        }
+        for (int j = 0; j < 4; ++j) enc_piece_v<BITS, W>(x[j], lo2, inv2, p[j]);
         if (ROTATED) enc_unrotate<W>(p, rot);
     } else {                                             // a flat group: every code is 0
 #pragma unroll
@@ -393,16 +450,7 @@ __device__ __forceinline__ void enc_group_v(const uint4 (&x)[4], int rot, uint32
 #pragma unroll
             for (int w = 0; w < W; ++w) p[j][w] = 0;
     }
-    if constexpr (BITS == 8) {
-        uint4 *o = reinterpret_cast<uint4 *>(codes_out);
-        o[0] = make_uint4(p[0][0], p[0][1], p[1][0], p[1][1]);
-        o[1] = make_uint4(p[2][0], p[2][1], p[3][0], p[3][1]);
-    }
-    if constexpr (BITS == 4)
-        *reinterpret_cast<uint4 *>(codes_out) = make_uint4(p[0][0], p[1][0], p[2][0], p[3][0]);
-    if constexpr (BITS == 2)
-        *reinterpret_cast<uint2 *>(codes_out) = make_uint2(__byte_perm(p[0][0], p[1][0], 0x5410),
-                                                           __byte_perm(p[2][0], p[3][0], 0x5410));
+    enc_store_group_v<BITS, W>(p, codes_out);
 }
 
 // Index, within the plane's V sections, of group gs of the tile's stage (stage rows hold cw / 32

@@ -83,21 +83,38 @@ __device__ __forceinline__ uint32_t tc_new_meta(uint32_t m, float &lo, float &sc
     return pack_bf16x2_rn(__fmaf_rn(0.0f, scale, lo), __fmaf_rn(qmax, scale, lo));      // xhat(0) | xhat(qmax) << 16
 }
 
-// One dequantised K row of a 4-channel column as two packed bf16 pairs.
-template <int BIN>
-__device__ __forceinline__ uint2 tc_row_k(const uint8_t *codes, const f32x2 (&lo)[2], const f32x2 (&sc)[2])
+// binary32 value of bf16_rne(x): the conversion of a pair whose other half is zero leaves exactly
+// that bit pattern (bf16 in the upper half, zeros below)
+__device__ __forceinline__ uint32_t round_to_bf16_bits(float x)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x), "f"(0.0f));
+    return r;
+}
+__device__ __forceinline__ f32x2 round_to_bf16(f32x2 v)
+{
+    uint32_t a, b;
+    f2_bits(v, a, b);
+    return f2_from_bits(round_to_bf16_bits(__uint_as_float(a)), round_to_bf16_bits(__uint_as_float(b)));
+}
+
+// One K row of a 4-channel column: unpack, dequantise, round to bf16 (the values stay binary32: no
+// packing and unpacking in between), quantise at the new level, store.
+template <int BIN, int BOUT>
+__device__ __forceinline__ void tc_row_k(const uint8_t *codes, const f32x2 (&lo)[2], const f32x2 (&sc)[2], f32x2 lo_a,
+                                         f32x2 lo_b, f32x2 inv_a, f32x2 inv_b, uint8_t *o)
 {
     f32x2 q[2];
     spread4<BIN>(codes, q);
-    uint32_t a, b, c2, d;
-    f2_bits(f2_fma(q[0], sc[0], lo[0]), a, b);
-    f2_bits(f2_fma(q[1], sc[1], lo[1]), c2, d);
-    return make_uint2(pack_bf16x2_rn(__uint_as_float(a), __uint_as_float(b)),
-                      pack_bf16x2_rn(__uint_as_float(c2), __uint_as_float(d)));
+    enc_store_row_k_f32<BOUT>(round_to_bf16(f2_fma(q[0], sc[0], lo[0])), round_to_bf16(f2_fma(q[1], sc[1], lo[1])), lo_a, lo_b,
+                              inv_a, inv_b, o);
 }
 
 // K: a thread owns 4 channels of one of the unit's tiles and walks that tile's rows (any number of
-// them).
+// them; a whole tile's 32 rows unrolled).  A channel stored flat at the new level has inv = 0 and
+// decoded values all equal to its min (its old range was below the threshold, or so large that the
+// new one overflowed: then its old scale was 0 as well), so value - min is 0 and the code 0 without
+// any masking.
 template <int BIN, int BOUT>
 __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int tid, uint64_t *empty_bar,
                                              int nt_unit, int tile0, int tpu, uint8_t *meta_sec, uint8_t *codes_sec)
@@ -112,15 +129,12 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int t
         const uint4 w4 = *reinterpret_cast<const uint4 *>(st + tc_meta_off(c * tpu) + 4 * (size_t)sub * c + 16 * (size_t)cq);
         const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
         float l1[4], s1[4], lo_new[4], inv[4];
-        uint32_t m[4], mask[4];
-        bool all_quantised = true;
+        uint32_t m[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             m[i] = tc_new_meta<BIN>(w[i], l1[i], s1[i]);
-            s1[i] = __fmul_rn(s1[i], Pos<BIN>::prescale(i));
+            if constexpr (BIN != 8) s1[i] = __fmul_rn(s1[i], Pos<BIN>::prescale(i));
             encode_params<BOUT>(m[i], lo_new[i], inv[i]);
-            mask[i] = inv[i] != 0.0f ? 0xffffffffu : 0u;
-            all_quantised = all_quantised && inv[i] != 0.0f;
         }
         uint4 *meta_out;
         uint8_t *out;
@@ -133,16 +147,14 @@ __device__ __forceinline__ void tc_consume_k(const uint8_t *st, RowGeom g, int t
         const f32x2 inv_a = f2_make(inv[0], inv[1]), inv_b = f2_make(inv[2], inv[3]);
         const uint32_t in_bytes = (uint32_t)c * BIN / 8;
         const uint8_t *src = st + (size_t)sub * kTileTokens * in_bytes + (size_t)cq * BIN / 2;   // 4 codes = BIN / 2 bytes
-        if (all_quantised) {
-#pragma unroll 8
-            for (int t = 0; t < nt; ++t)
-                enc_store_row_k<BOUT, false>(tc_row_k<BIN>(src + (size_t)t * in_bytes, lo, sc), lo_a, lo_b, inv_a, inv_b,
-                                             mask, out + (size_t)t * out_bytes);
+        if (nt == kTileTokens) {
+#pragma unroll
+            for (int t = 0; t < kTileTokens; ++t)
+                tc_row_k<BIN, BOUT>(src + (size_t)t * in_bytes, lo, sc, lo_a, lo_b, inv_a, inv_b, out + (size_t)t * out_bytes);
         } else {
 #pragma unroll 1
             for (int t = 0; t < nt; ++t)
-                enc_store_row_k<BOUT, true>(tc_row_k<BIN>(src + (size_t)t * in_bytes, lo, sc), lo_a, lo_b, inv_a, inv_b,
-                                            mask, out + (size_t)t * out_bytes);
+                tc_row_k<BIN, BOUT>(src + (size_t)t * in_bytes, lo, sc, lo_a, lo_b, inv_a, inv_b, out + (size_t)t * out_bytes);
         }
     }
     enc_release(empty_bar);
@@ -158,23 +170,31 @@ __device__ __forceinline__ void tc_consume_v(const uint8_t *st, RowGeom geom, in
     uint32_t *meta = reinterpret_cast<uint32_t *>(meta_sec);
     const f32x2 pre01 = f2_make(Pos<BIN>::prescale(0), Pos<BIN>::prescale(1));
     const f32x2 pre23 = f2_make(Pos<BIN>::prescale(2), Pos<BIN>::prescale(3));
+    constexpr int W = BOUT == 8 ? 2 : 1;
 #pragma unroll 2
     for (int g = tid; g < ngroups; g += kEncGroupThreads) {
-        float l1, s0;
+        float l1, s0, lo_new, inv;
         const uint32_t m = tc_new_meta<BIN>(meta_in[g], l1, s0);
+        encode_params<BOUT>(m, lo_new, inv);
         const f32x2 ss = f2_make(s0, s0), ll = f2_make(l1, l1);
-        const f32x2 sa = f2_mul(ss, pre01), sb = f2_mul(ss, pre23);          // exact: powers of two
-        const f32x2 sc[4] = {sa, sb, sa, sb}, lo[4] = {ll, ll, ll, ll};
+        f32x2 sa = ss, sb = ss;
+        if constexpr (BIN != 8) { sa = f2_mul(ss, pre01); sb = f2_mul(ss, pre23); }     // exact: powers of two
+        const f32x2 sc[4] = {sa, sb, sa, sb};
+        const f32x2 lo2 = f2_make(lo_new, lo_new), inv2 = f2_make(inv, inv);
         const uint8_t *src = st + (size_t)g * (4 * BIN);  // 32 codes = 4 * BIN bytes
-        uint4 x[4];
+        uint32_t p[4][W];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            f32x2 q[4];
+            // a group stored flat at the new level decodes to its min everywhere: value - min = 0, code 0
+            f32x2 q[4], x[4];
             spread8<BIN>(src + j * BIN, q);
-            x[j] = fma_pack8(q, sc, lo);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) x[k] = round_to_bf16(f2_fma(q[k], sc[k], ll));
+            enc_piece_v_f32<BOUT, W>(x, lo2, inv2, p[j]);
         }
         const size_t gi = enc_v_group_index(geom, tile, g);
-        enc_group_v<BOUT, false>(x, 0, m, meta + gi, codes_sec + gi * (4 * BOUT));
+        meta[gi] = m;
+        enc_store_group_v<BOUT, W>(p, codes_sec + gi * (4 * BOUT));
     }
     enc_release(empty_bar);
 }
