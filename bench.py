@@ -498,10 +498,13 @@ def time_extras(kvh, w, reps: int = 5):
 
 def mix_ceiling(w, reps: int = 10):
     """What kernels that do no codec work reach at the read : write mix of each level's decode
-    launch, on the same amount of data: a plain grid-stride loop of 16-byte loads and stores, and a
-    loop of bulk copies through shared memory (no per-element instructions at all).  Not bounds,
-    but they show how much of a level's distance from the copy peak belongs to the memory system's
-    handling of write-heavy streams."""
+    launch, on the same amount of data: a plain grid-stride loop of 16-byte loads and stores, a
+    loop of bulk copies through shared memory (no per-element instructions at all; with a fixed
+    stride and with units handed out dynamically), and the decode
+    kernel's own skeleton (producer warp, two-stage ring, 8 consumer warps, dynamic hand-out of
+    units, the same store pattern) with the codec taken out.  Not bounds, but they show how much of
+    a level's distance from the copy peak belongs to the memory system's handling of write-heavy
+    streams, and the last one what the arithmetic costs on top of moving the bytes."""
     import ctypes
     from paper_2509_00105_b200 import _build
     L = ctypes.CDLL(str(_build.build(variant="probe")))
@@ -514,9 +517,9 @@ def mix_ceiling(w, reps: int = 10):
         if leg.level is None:
             continue
         reads16 = {0: 16, 1: 9, 2: 5, 3: 3}[leg.level]           # 16-byte reads per 16 16-byte writes
-        write_bytes = (2 * leg.elements) // 16384 * 16384
+        write_bytes = (2 * leg.elements) // 65536 * 65536
         row = {"level": leg.level, "read_write": f"{reads16}:16"}
-        for kind, name in ((0, "ldst"), (1, "bulk")):
+        for kind, name in ((0, "ldst"), (1, "bulk"), (3, "bulk_dyn"), (2, "ring")):
             def fn():
                 st = L.kvh_probe_stream_mix(kind, w.kv.data_ptr(), dst.data_ptr(), write_bytes, reads16,
                                             w.status.data_ptr(), torch.cuda.current_stream().cuda_stream)
