@@ -502,7 +502,8 @@ def mix_ceiling(w, reps: int = 10):
     loop of bulk copies through shared memory (no per-element instructions at all; with a fixed
     stride and with units handed out dynamically), and the decode
     kernel's own skeleton (producer warp, two-stage ring, 8 consumer warps, dynamic hand-out of
-    units, the same store pattern) with the codec taken out.  Not bounds, but they show how much of
+    units, the same store pattern) with the codec taken out, writing its pages in order and to
+    pseudo-random pages of the destination as a shuffled page table makes the decoder do.  Not bounds, but they show how much of
     a level's distance from the copy peak belongs to the memory system's handling of write-heavy
     streams, and the last one what the arithmetic costs on top of moving the bytes."""
     import ctypes
@@ -519,7 +520,7 @@ def mix_ceiling(w, reps: int = 10):
         reads16 = {0: 16, 1: 9, 2: 5, 3: 3}[leg.level]           # 16-byte reads per 16 16-byte writes
         write_bytes = (2 * leg.elements) // 65536 * 65536
         row = {"level": leg.level, "read_write": f"{reads16}:16"}
-        for kind, name in ((0, "ldst"), (1, "bulk"), (3, "bulk_dyn"), (2, "ring")):
+        for kind, name in ((0, "ldst"), (1, "bulk"), (3, "bulk_dyn"), (2, "ring"), (4, "ring_scatter")):
             def fn():
                 st = L.kvh_probe_stream_mix(kind, w.kv.data_ptr(), dst.data_ptr(), write_bytes, reads16,
                                             w.status.data_ptr(), torch.cuda.current_stream().cuda_stream)

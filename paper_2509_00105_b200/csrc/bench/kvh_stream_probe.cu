@@ -13,6 +13,8 @@
 //           cluster launch control, three CTAs per SM; per unit a consumer thread loads 16 bytes from
 //           the stage per row and stores them as one 16-byte vector of each of its 16 (or 8) rows of
 //           2 KiB, the decode kernel's store pattern, and does nothing else
+//   kind 4  kind 2 writing every 32 KiB page (16 rows of 2 KiB, a 16-token page of one plane) to a
+//           pseudo-random page of the destination: what a shuffled page table does to the store stream
 //   kind 3  kind 1 with its units handed out through cluster launch control instead of a fixed
 //           stride (SMs do not all reach memory equally fast, so a fixed stride waits for the slowest)
 #include <cuda_runtime.h>
@@ -181,7 +183,12 @@ constexpr uint32_t kRingStageBytes = 36u * 1024u;                 // the decode 
 constexpr uint32_t kRingRowBytes = 2048u;                         // a page row of 1024 bf16 channels
 
 // ROWS: rows of 2 KiB a thread writes per unit (16: 64 KiB per unit; 8: 32 KiB, the raw level's half tile)
-template <int ROWS>
+// SCATTER: the destination's 32 KiB pages are permuted (page i of the sequential order goes to page
+// i * 104729 mod n_pages; the multiplier shares no factor with the page counts used here, so this is
+// a bijection).
+constexpr uint32_t kRingPage = 32u * 1024u;
+constexpr uint64_t kRingScatterMul = 104729ull;
+template <int ROWS, bool SCATTER>
 __global__ void __launch_bounds__(kRingThreads, 3) ring_mix_kernel(const uint8_t *__restrict__ src, uint8_t *__restrict__ dst,
                                                                    uint32_t n_units, uint32_t in_bytes, int32_t *status)
 {
@@ -266,7 +273,12 @@ __global__ void __launch_bounds__(kRingThreads, 3) ring_mix_kernel(const uint8_t
             const int64_t id = unit_of[s];
             if (id < 0) break;
             const uint4 *st = reinterpret_cast<const uint4 *>(stage_mem + (size_t)s * kRingStageBytes);
-            uint4 *out = reinterpret_cast<uint4 *>(dst + (uint64_t)id * kUnitWrite + (size_t)g * ROWS * kRingRowBytes) + cv;
+            uint64_t off = (uint64_t)id * kUnitWrite + (uint64_t)g * ROWS * kRingRowBytes;    // a thread's rows lie in one page
+            if (SCATTER) {
+                const uint64_t n_pages = (uint64_t)n_units * kUnitWrite / kRingPage;
+                off = (off / kRingPage * kRingScatterMul) % n_pages * kRingPage + off % kRingPage;
+            }
+            uint4 *out = reinterpret_cast<uint4 *>(dst + off) + cv;
             uint32_t v = threadIdx.x;                            // < 256 <= n_vec
 #pragma unroll
             for (int k = 0; k < ROWS; ++k) {
@@ -292,10 +304,10 @@ kvh_status launch_ldst(const void *src, void *dst, uint64_t n_units, int sms, cu
 
 }  // namespace
 
-// kind: 0 .. 3 (see above).  src [device, 16-byte aligned]: at least write_bytes * reads16 / 16 bytes;
+// kind: 0 .. 4 (see above).  src [device, 16-byte aligned]: at least write_bytes * reads16 / 16 bytes;
 // dst [device, 16-byte aligned]: write_bytes, a multiple of 16 KiB; reads16 in {16, 9, 5, 3}: 16-byte
 // reads per 16 16-byte writes (the decode mixes of levels 0..3).  dev_status [device]: receives
-// KVH_ERR_TIMEOUT if a bounded wait inside kinds 1 to 3 runs out; kind 2 wants write_bytes to be a
+// KVH_ERR_TIMEOUT if a bounded wait inside kinds 1 to 4 runs out; kinds 2 and 4 want write_bytes to be a
 // multiple of 64 KiB.  Returns once the launch is enqueued.
 extern "C" kvh_status kvh_probe_stream_mix(int kind, const void *src, void *dst, uint64_t write_bytes, int reads16,
                                            int32_t *dev_status, void *stream)
@@ -317,7 +329,7 @@ extern "C" kvh_status kvh_probe_stream_mix(int kind, const void *src, void *dst,
         default: return KVH_ERR_INVALID_ARG;
         }
     }
-    if (kind == 2) {
+    if (kind == 2 || kind == 4) {
         if (reads16 != 16 && reads16 != 9 && reads16 != 5 && reads16 != 3) return KVH_ERR_INVALID_ARG;
         // the raw level is fed in half tiles (32 KiB in, 32 KiB out), the quantised ones in whole tiles
         const bool half = reads16 == 16;
@@ -326,7 +338,10 @@ extern "C" kvh_status kvh_probe_stream_mix(int kind, const void *src, void *dst,
         const uint32_t n_units = (uint32_t)(write_bytes / unit_write);
         const uint32_t in_bytes = unit_write / 16u * (uint32_t)reads16;
         const size_t dyn = (size_t)kRingStages * kRingStageBytes;
-        auto kernel = half ? ring_mix_kernel<8> : ring_mix_kernel<16>;
+        const uint64_t n_pages = write_bytes / kRingPage;
+        if (kind == 4 && n_pages % kRingScatterMul == 0) return KVH_ERR_INVALID_ARG;   // the multiplier is prime: a bijection otherwise
+        auto kernel = kind == 4 ? (half ? ring_mix_kernel<8, true> : ring_mix_kernel<16, true>)
+                                : (half ? ring_mix_kernel<8, false> : ring_mix_kernel<16, false>);
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) != cudaSuccess)
             return KVH_ERR_CUDA;
         kernel<<<n_units, kRingThreads, dyn, st>>>(static_cast<const uint8_t *>(src), static_cast<uint8_t *>(dst), n_units,

@@ -48,13 +48,11 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
             return KVH_ERR_CUDA;
-        const uint32_t stage = tma_stage_bytes(p.bw * p.tpu);
-        // 72 KiB of stages per CTA: three CTAs (24 consumer warps) per SM, two stages each when
-        // c = 1024.  Measured against three stages and two CTAs per SM: the same at levels 0 and 1, 2-4 %
-        // faster at levels 2 and 3, where the consumers are short of issue slots rather than of data.
-        int stages = (int)((72u * 1024u) / stage);
-        stages = stages < 2 ? 2 : (stages > kMaxStages ? kMaxStages : stages);
-        const size_t dyn = (size_t)stages * stage;
+        // Stage memory per CTA: a ring of quanta of 12 * c bytes, 72 KiB of them when c = 1024, so
+        // that three CTAs (24 consumer warps) share an SM.  A unit takes 1, 2 or 3 quanta by its
+        // level: 6 units in flight at 2 bits, 3 at 4 bits, 2 at 8 bits or raw.
+        const int quanta = ring_quanta(p.bw * p.tpu);
+        const size_t dyn = (size_t)quanta * tma_quantum_bytes(p.bw * p.tpu);
         // the instance with the channel count of the Llama-3 shapes compiled in, or the general one
         auto kernel = p.c == 1024 ? (small_pages ? decode_tma_kernel<1024, true> : decode_tma_kernel<1024, false>)
                                   : (small_pages ? decode_tma_kernel<0, true> : decode_tma_kernel<0, false>);
@@ -65,7 +63,7 @@ kvh_status launch_decode(DecodeParams &p, const kvh_pool *pool, int n_chunks, vo
         const int sched = kTileSched;
         const int64_t resident = (int64_t)sms * per_sm;
         const unsigned pgrid = sched == 1 ? (unsigned)tiles : (unsigned)(tiles < resident ? tiles : resident);
-        kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, stages, sched);
+        kernel<<<pgrid, kTmaThreads, dyn, static_cast<cudaStream_t>(stream)>>>(p, n_chunks, quanta, sched);
         return launch_status();
     }
     decode_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);

@@ -9,11 +9,16 @@
 // in flight while the current one is being expanded, so HBM latency is off the critical path and
 // the kernel runs at the speed of its writes (2 of the (b+1)/8 + 2 bytes moved per element).
 //
-// A unit is a 32-token tile of a quantised plane (<= 32*c bytes of codes + 4*c bytes of metadata)
-// or one 16-token half of a raw bf16 tile (32*c bytes), so every unit fits one stage.  Rows of at
-// most 512 channels would leave threads idle and make units small, so there a unit takes 2, 4 or 8
-// consecutive tiles of the plane (DecodeParams::tpu; codes and metadata of consecutive tiles are
-// contiguous in the stream) and the stage grows by the same factor.
+// A unit is a 32-token tile of a quantised plane (32*c*b/8 bytes of codes + 4*c bytes of metadata)
+// or one 16-token half of a raw bf16 tile (32*c bytes).  Rows of at most 512 channels would leave
+// threads idle and make units small, so there a unit takes 2, 4 or 8 consecutive tiles of the plane
+// (DecodeParams::tpu; codes and metadata of consecutive tiles are contiguous in the stream).
+//
+// Stages are cut from a ring of quanta of 12*c bytes, as many per unit as its level needs: one at
+// 2 bits, two at 4 bits, three at 8 bits and for a raw half tile.  With the 72 KiB a CTA has at
+// c = 1024 that is 6 units in flight at 2 bits, 3 at 4 bits and 2 at 8 bits or raw, whatever the
+// mix of levels in the launch.  The kernel is bound by memory and its CTAs by the latency of their
+// copies, so the more bytes a CTA has on their way, the less often its consumers stand idle.
 //
 // Every wait is bounded: a wait that runs out reports KVH_ERR_TIMEOUT, raises the CTA's abort
 // flag and the CTA leaves after its copies in flight have landed.
@@ -27,7 +32,8 @@ namespace kvh {
 
 constexpr int kConsumerThreads = 256;
 constexpr int kTmaThreads = kConsumerThreads + 32;      // + one producer warp
-constexpr int kMaxStages = 8;
+constexpr int kSlots = 8;                               // units a CTA can have between producer and consumers
+constexpr int kMaxQuanta = 24;
 constexpr int kTmaMaxChannels = 1024;
 
 struct UnitInfo {
@@ -39,9 +45,21 @@ struct UnitInfo {
     const int32_t *pgs;  // the same and up to 12 more, in shared memory (units of several tiles)
     uint16_t *plane;     // pool + layer*layer_stride + kv*kv_stride
     int32_t col0, cw;    // first channel and width of the unit's column block (0, c unless rows exceed 1024 channels)
+    uint32_t st_off;     // where the unit's codes (or raw rows) start in the CTA's stage memory
+    uint32_t meta_off;   // its metadata, from there
 };
 
-__host__ __device__ __forceinline__ uint32_t tma_stage_bytes(int c) { return (36u * (uint32_t)c + 127u) & ~127u; }
+// One quantum of stage memory, for units of c channels (times the tiles a unit holds): the codes of a
+// 32-token tile at 2 bits (8*c bytes) and its metadata (4*c bytes).
+__host__ __device__ __forceinline__ uint32_t tma_quantum_bytes(int c) { return (12u * (uint32_t)c + 127u) & ~127u; }
+// Quanta a unit takes: its codes (bits 2, 4, 8) or raw rows (16: half a tile) plus 4*c bytes of metadata.
+__host__ __device__ __forceinline__ int unit_quanta(int bits) { return bits == 0 ? 0 : bits == 2 ? 1 : bits == 4 ? 2 : 3; }
+// Quanta of a CTA's ring: what 72 KiB hold (three CTAs per SM), at least the 6 that let any unit in.
+__host__ __device__ __forceinline__ int ring_quanta(int c)
+{
+    const int q = (int)((72u * 1024u) / tma_quantum_bytes(c));
+    return q < 6 ? 6 : (q > kMaxQuanta ? kMaxQuanta : q);
+}
 __host__ __device__ __forceinline__ uint32_t round16(uint32_t x) { return (x + 15u) & ~15u; }
 
 // ---- dequantisation of 8 consecutive codes with few instructions per element ----------------
@@ -394,25 +412,24 @@ __device__ __forceinline__ void consume_v_full(const DecodeParams &p, const Unit
 //            launch control, so faster SMs take more tiles.
 template <int C, bool SMALLPG = false>
 __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const DecodeParams p, const int n_chunks,
-                                                                 const int n_stages, const int sched)
+                                                                 const int n_quanta, const int sched)
 {
     extern __shared__ __align__(128) uint8_t stage_mem[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
-    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-    __shared__ UnitInfo info[kMaxStages];
-    __shared__ int32_t unit_pg[kMaxStages][16];
+    __shared__ __align__(8) uint64_t full_bar[kSlots];
+    __shared__ __align__(8) uint64_t empty_bar[kSlots];
+    __shared__ UnitInfo info[kSlots];
+    __shared__ int32_t unit_pg[kSlots][16];
     __shared__ int abort_flag;
     __shared__ int wait_verdict[2];
     __shared__ __align__(16) uint4 clc_response[2];
     __shared__ __align__(8) uint64_t clc_bar[2];
 
     const int tpu = C ? 1 : p.tpu;                        // tiles per unit
-    const uint32_t stage_bytes = tma_stage_bytes(p.bw * tpu);
-    const uint32_t meta_off = 32u * p.bw * tpu;
+    const uint32_t quantum = tma_quantum_bytes(p.bw * tpu);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < n_stages; ++s) {
+        for (int s = 0; s < kSlots; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerThreads / 32);
         }
@@ -434,6 +451,12 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
         LayerLayout L = layer_layout(0, p.c, 1);
         uint32_t unit = 0;
         bool ok = true;
+        // The ring of quanta: units take their quanta at head_q, in order, never across the ring's end
+        // (the quanta left before the end are given up with the unit that did not fit there), and hand
+        // them back in the same order when the consumers release them.  tail is the oldest unit whose
+        // quanta have not been taken back; lane j remembers what the unit in slot j holds.
+        uint32_t tail = 0;
+        int head_q = 0, free_q = n_quanta, slot_q = 0;
 
         // One unit.  Contiguous source (rows as wide as the plane): one copy of codes_bytes and one of
         // meta_bytes.  A column block of wider rows (row_stride != 0): lane r copies row r's codes_bytes
@@ -442,13 +465,25 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
         auto emit = [&](int bits, int kv, int row0, int nrows, uint16_t *plane, int col0, const uint8_t *codes_src,
                         uint32_t codes_bytes, uint32_t row_stride, const uint8_t *meta_src, uint32_t meta_bytes,
                         uint32_t mrow_stride) -> bool {
-            const int s = unit % n_stages;
-            if (unit >= (uint32_t)n_stages) {
+            const int s = unit % kSlots;
+            const int need = unit_quanta(bits);
+            const int pad = head_q + need > n_quanta ? n_quanta - head_q : 0;
+            while (unit - tail >= (uint32_t)kSlots || free_q < need + pad) {
+                if (tail == unit) return false;              // nothing left to take back: cannot happen (the ring holds any unit)
                 bool w = true;
-                if (lane == 0) w = mbar_wait(&empty_bar[s], ((unit / n_stages) - 1) & 1, &abort_flag);
+                if (lane == 0) w = mbar_wait(&empty_bar[tail % kSlots], (tail / kSlots) & 1, &abort_flag);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) return false;
+                free_q += __shfl_sync(0xffffffffu, slot_q, tail % kSlots);
+                ++tail;
             }
+            if (pad) head_q = 0;
+            const uint32_t st_off = (uint32_t)head_q * quantum;
+            const uint32_t meta_off = 4u * (uint32_t)(bits == 16 ? 8 : bits) * p.bw * tpu;   // behind a tile's codes
+            head_q += need;
+            if (head_q == n_quanta) head_q = 0;
+            free_q -= need + pad;
+            if (lane == s) slot_q = need + pad;
             const int pidx = row0 >> p.page_shift;
             int32_t pg[4];
 #pragma unroll
@@ -456,13 +491,14 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
             const int32_t pg_mine = __shfl_sync(0xffffffffu, my_pg, (pidx + lane) & 31);
             if (lane < 16) unit_pg[s][lane] = pg_mine;
             __syncwarp();                                // lane 0's arrival below publishes these too
-            uint8_t *st = stage_mem + (size_t)s * stage_bytes;
+            uint8_t *st = stage_mem + st_off;
             const bool strided = row_stride != 0;
             if (lane == 0) {
                 UnitInfo &u = info[s];
                 u.bits = bits; u.kv = kv; u.row0 = row0; u.nrows = nrows; u.plane = plane;
                 u.pg[0] = pg[0]; u.pg[1] = pg[1]; u.pg[2] = pg[2]; u.pg[3] = pg[3];
                 u.col0 = col0; u.cw = p.bw;
+                u.st_off = st_off; u.meta_off = meta_off;
                 if (bits == 0) {
                     mbar_arrive(&full_bar[s]);
                 } else if (!strided) {
@@ -490,13 +526,22 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share page rows
-            const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
-            const int64_t plane_id = row_tile / upc;
+            // a tile id fits 32 bits (the host refuses larger launches): unsigned 32-bit divisions, and none
+            // but the one by the layer count when the row width is compiled in.  The producer's arithmetic
+            // is serial code in one warp and sits between a stage coming free and the next copy's start.
+            const uint32_t id = (uint32_t)tile_id;
+            const uint32_t nb = C ? 1u : (uint32_t)p.n_blocks, units = C ? (uint32_t)kTilesPerChunk : (uint32_t)upc;
+            const int cb = (int)(id % nb);                       // column block, fastest: neighbours share page rows
+            const uint32_t row_tile = id / nb;
+            const int tile = (int)(row_tile % units) * tpu;      // the unit's first tile
+            // Order of the tiles: a chunk's tiles, then the chunks, then the (layer, K|V) planes.  CTAs that
+            // run side by side thus write into one plane of the pool (pages scattered over 64 MiB, not over
+            // the whole pool: the same few translations serve every SM) and read from neighbouring chunks.
+            const uint32_t t2 = row_tile / units;
+            const int chunk = (int)(t2 % (uint32_t)n_chunks);
+            const uint32_t plane_id = t2 / (uint32_t)n_chunks;
             const int kv = (int)(plane_id & 1);
-            const int layer = (int)((plane_id >> 1) % p.l);
-            const int chunk = (int)((plane_id >> 1) / p.l);
+            const int layer = (int)(plane_id >> 1);
             if (chunk != cur_chunk) {
                 cur_chunk = chunk;
                 if (p.descs) d = p.descs[chunk];
@@ -565,27 +610,26 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
             abort_flag = 1;
         }
         // Leave only after every copy issued has landed: a normal run has seen them all consumed;
-        // after an abort the last n_stages units may still be in flight.
+        // after an abort the units not taken back yet may still be in flight.
         if (lane == 0) {
             int never = 0;                           // the drain ignores the abort flag
-            const uint32_t first = unit > (uint32_t)n_stages ? unit - n_stages : 0;
-            for (uint32_t w = first; w < unit; ++w)
-                (void)mbar_wait(&full_bar[w % n_stages], (w / n_stages) & 1, &never);
+            for (uint32_t w = tail; w < unit; ++w)
+                (void)mbar_wait(&full_bar[w % kSlots], (w / kSlots) & 1, &never);
             feed.drain();
         }
     } else {
         // ------------------------------ consumer warps ------------------------------
         for (uint32_t unit = 0;; ++unit) {
-            const int s = unit % n_stages;
-            if (!group_wait(&full_bar[s], (unit / n_stages) & 1, &abort_flag, wait_verdict, unit, 1, kConsumerThreads, warp == 0)) {
+            const int s = unit % kSlots;
+            if (!group_wait(&full_bar[s], (unit / kSlots) & 1, &abort_flag, wait_verdict, unit, 1, kConsumerThreads, warp == 0)) {
                 if (threadIdx.x == 0) report(p.status, KVH_ERR_TIMEOUT);
                 break;
             }
             UnitInfo u = info[s];
             if (u.bits == 0) break;
             u.pgs = unit_pg[s];
-            const uint8_t *st = stage_mem + (size_t)s * stage_bytes;
-            const uint8_t *mt = st + meta_off;
+            const uint8_t *st = stage_mem + u.st_off;
+            const uint8_t *mt = st + u.meta_off;
             bool done = false;
             if constexpr (C != 0 && !SMALLPG) {
                 // the common case by far: a whole tile (or, raw, a whole 16-token half of one)

@@ -590,13 +590,16 @@ encode_tma_kernel(const EncodeParams p, const int n_chunks, const int sched, con
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int cb = (int)(tile_id % p.n_blocks);          // column block, fastest: neighbours share rows
-            const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
-            const int64_t plane_id = row_tile / upc;
+            // a tile id fits 32 bits (the host refuses larger launches): unsigned 32-bit divisions
+            const uint32_t id = (uint32_t)tile_id;
+            const uint32_t nb = (uint32_t)p.n_blocks, units = (uint32_t)upc;
+            const int cb = (int)(id % nb);                       // column block, fastest: neighbours share rows
+            const uint32_t row_tile = id / nb;
+            const int tile = (int)(row_tile % units) * tpu;      // the unit's first tile
+            const uint32_t plane_id = row_tile / units;
             const int kv = (int)(plane_id & 1);
-            const int layer = (int)((plane_id >> 1) % p.l);
-            const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), p.chunk0);
+            const int layer = (int)((plane_id >> 1) % (uint32_t)p.l);
+            const int chunk = chunks.chunk((int)((plane_id >> 1) / (uint32_t)p.l), p.chunk0);
             const int64_t tok0 = (int64_t)chunk * kChunkTokens;
             const int n_expect = (int)min((int64_t)kChunkTokens, p.N - tok0);
             kvh_chunk_desc d;

@@ -299,13 +299,16 @@ transcode_tma_kernel(const TranscodeParams p, const int n_chunks, const int sche
         };
 
         auto do_tile = [&](int64_t tile_id) {
-            const int cb = (int)(tile_id % p.n_blocks);          // column block (rows wider than 1024 channels)
-            const int64_t row_tile = tile_id / p.n_blocks;
-            const int tile = (int)(row_tile % upc) * tpu;        // the unit's first tile
-            const int64_t plane_id = row_tile / upc;
+            // a tile id fits 32 bits (the host refuses larger launches): unsigned 32-bit divisions
+            const uint32_t id = (uint32_t)tile_id;
+            const uint32_t nb = (uint32_t)p.n_blocks, units = (uint32_t)upc;
+            const int cb = (int)(id % nb);                       // column block (rows wider than 1024 channels)
+            const uint32_t row_tile = id / nb;
+            const int tile = (int)(row_tile % units) * tpu;      // the unit's first tile
+            const uint32_t plane_id = row_tile / units;
             const int kv = (int)(plane_id & 1);
-            const int layer = (int)((plane_id >> 1) % p.l);
-            const int chunk = chunks.chunk((int)((plane_id >> 1) / p.l), 0);
+            const int layer = (int)((plane_id >> 1) % (uint32_t)p.l);
+            const int chunk = chunks.chunk((int)((plane_id >> 1) / (uint32_t)p.l), 0);
             if (chunk != cur_chunk) {
                 cur_chunk = chunk;
                 di = p.in_descs[chunk];
