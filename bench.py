@@ -74,11 +74,16 @@ WORKLOAD_NAMES = ["tiny", "llama3-8b-8k", BATCH, "llama3-70b-32k", "llama3-8b-12
 # kernel sources with the digest recorded beside them (kernel_source_digest()); once a kernel source
 # has changed, `traffic` is reported as null until the capture is repeated.
 TRAFFIC = {
-    "captured": "2026-11-27",
-    "source_digest": "",
-    "decode": {0: 0.981, 1: 0.973, 2: 0.967, 3: 0.964},
-    "encode": {0: 0.979, 1: 0.979, 2: 0.986, 3: 0.992},
+    "captured": "2026-11-28",
+    "source_digest": "c42eb9dbd588ee6f",
+    "decode": {0: 0.9808, 1: 0.9725, 2: 0.9667, 3: 0.9635},
+    "encode": {0: 0.9792, 1: 0.9786, 2: 0.9865, 3: 0.9921},
+    # executed thread instructions per element of the transcoding instances whose source is quantised
+    # (smsp__inst_executed.sum x 32 / elements of the same capture): these are bound by instruction
+    # issue, not by memory
+    "transcode_instr": {(1, 2): 8.22, (1, 3): 8.24, (2, 3): 8.42},
 }
+ISSUE_LANES_PER_SM = 4 * 32      # four schedulers per SM, one warp instruction (32 threads) per clock each
 
 
 def kernel_source_digest() -> str:
@@ -147,6 +152,15 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        note = None
+        if not self.lines:                               # the region was shorter than one sampling period: one reading now
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-i", self.gpu],
+                                     capture_output=True, text=True, timeout=10).stdout
+                self.lines = out.splitlines()
+                note = "timed region shorter than the sampling period: one reading taken right after it"
+            except (OSError, subprocess.TimeoutExpired):
+                pass
         sm, mx, power, reasons = [], [], [], set()
         for line in self.lines:
             p = [x.strip() for x in line.split(",")]
@@ -159,8 +173,11 @@ class ClockSampler:
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+               "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        if note:
+            out["note"] = note
+        return out
 
 
 class NvmlClock:
@@ -457,20 +474,24 @@ def level_statistics(w, clock: NvmlClock, reps: int, flush, peak: float) -> list
     return out
 
 
-def time_extras(kvh, w, reps: int = 5):
+def time_extras(kvh, w, clock: "NvmlClock", sms: int, instr_ok: bool, reps: int = 20):
     """Transcoding (every pair of levels) and token dropping (4 sink tokens + a recent window, a
     quarter of the context kept), each as the mean of `reps` launches over the whole context after
     one warm-up launch.  Bytes counted: streams read + streams written (transcode), kept bf16 rows
-    read + streams written (token dropping)."""
+    read + streams written (token dropping).  Transcoding from a quantised source is bound by
+    instruction issue: its line carries an "alu" roofline too, the time the counted thread
+    instructions per element need at one warp instruction per scheduler and clock, at the SM clock
+    sampled during the launches."""
     def timed(fn):
         fn()
+        clock.start()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(reps):
             fn()
         b.record()
         b.synchronize()
-        return a.elapsed_time(b) / reps
+        return a.elapsed_time(b) / reps, clock.stop()
 
     l, c, N = w.l, w.c, w.N
     elements = l * 2 * N * c
@@ -481,15 +502,22 @@ def time_extras(kvh, w, reps: int = 5):
         kvh.encode(w.kv, lin, out=w.stream_buf[:total_in], dev_status=w.status)
         for lout in range(lin + 1, 4):
             _, descs_out_dev, total_out = w.plans[lout]
-            ms = timed(lambda: kvh.transcode(w.stream_buf[:total_in], descs_in_dev, second[:total_out], descs_out_dev,
-                                             w.n_chunks, l, c, lin, lout, dev_status=w.status))
-            out["transcode"].append({"from": lin, "to": lout, "ms": round(ms, 4),
-                                     "hbm_gbps": round((total_in + total_out) / ms / 1e6, 1),
-                                     "tokens_per_s": round(N / ms * 1e3)})
+            ms, mhz = timed(lambda: kvh.transcode(w.stream_buf[:total_in], descs_in_dev, second[:total_out], descs_out_dev,
+                                                  w.n_chunks, l, c, lin, lout, dev_status=w.status))
+            row = {"from": lin, "to": lout, "ms": round(ms, 4), "hbm_gbps": round((total_in + total_out) / ms / 1e6, 1),
+                   "tokens_per_s": round(N / ms * 1e3)}
+            per_el = TRAFFIC["transcode_instr"].get((lin, lout))
+            if per_el and instr_ok and mhz:
+                bound_ms = elements * per_el / (sms * ISSUE_LANES_PER_SM * mhz * 1e3)
+                row["roofline_alu"] = {"bound": "alu", "thread_instr_per_element": per_el, "sm_mhz": mhz,
+                                       "peak": round(sms * ISSUE_LANES_PER_SM * mhz / 1e6, 2), "unit": "T thread-instr/s",
+                                       "achieved": round(elements * per_el / ms / 1e9, 2), "bound_ms": round(bound_ms, 4),
+                                       "frac": round(bound_ms / ms, 4)}
+            out["transcode"].append(row)
     runs, n_kept = kvh.keep_sinks_and_recent(N, 4, max(N // 4 - 4, 1))
     for level in LEVELS:
         descs, total = kvh.plan_chunks(l, c, n_kept, level)
-        ms = timed(lambda: kvh.encode_kept(w.kv, runs, None, len(descs), second[:total], w.status, level=level))
+        ms, _ = timed(lambda: kvh.encode_kept(w.kv, runs, None, len(descs), second[:total], w.status, level=level))
         out["token_dropping"].append({"level": level, "kept_tokens": n_kept, "ms": round(ms, 4),
                                       "hbm_gbps": round((2 * elements * n_kept // N + total) / ms / 1e6, 1)})
     assert w.status.item() == 0
@@ -618,7 +646,9 @@ def run_ours(args):
     # ---- the two further store-side operations and the plain-streaming ceilings ----
     extras = None
     if single and not args.no_extras and isinstance(w, ContextWorkload):
-        extras = time_extras(kvh, w)
+        sms = torch.cuda.get_device_properties(local).multi_processor_count
+        extras = time_extras(kvh, w, NvmlClock(bus), sms, TRAFFIC["source_digest"] == kernel_source_digest() and w.c == 1024,
+                             reps=args.extras_reps)
         extras["mix_ceiling"] = mix_ceiling(w)
 
     # ---- end to end: stored form in pinned host memory ----
@@ -789,6 +819,7 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="shorten the context (profiling only; not a bench line)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--stat-launches", type=int, default=50, help="launches per level and direction in level_stats; 0 skips")
+    ap.add_argument("--extras-reps", type=int, default=20, help="launches per transcode pair / token-dropping level in extras")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the transcode / token-dropping / mix-ceiling timings")
@@ -800,7 +831,8 @@ def main():
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(relaunch_as_ranks(args.gpus))
     if args.steps is None:
-        args.steps = {"tiny": 200, BATCH: 20}.get(args.workload, 50)
+        # timed region of about half a second or more, so that the clock sampler sees it
+        args.steps = {"tiny": 1000, "llama3-8b-8k": 300, BATCH: 20}.get(args.workload, 50)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.tokens and args.workload == BATCH:
         ap.error("--tokens applies to the single-context workloads")
