@@ -514,6 +514,15 @@ def time_extras(kvh, w, clock: "NvmlClock", sms: int, instr_ok: bool, reps: int 
                                        "achieved": round(elements * per_el / ms / 1e9, 2), "bound_ms": round(bound_ms, 4),
                                        "frac": round(bound_ms / ms, 4)}
             out["transcode"].append(row)
+    # a level per chunk (uniformly random): the general encoder instance over device descriptors alone, and the
+    # per-level instances when the caller also passes its host copy of the descriptors
+    lv = workloads.chunk_levels(w.n_chunks, 4, seed=77)
+    mdescs, mtotal = kvh.plan_chunks(l, c, N, lv)
+    mdev = kvh.descs_to_tensor(mdescs, w.dev)
+    out["encode_mixed_levels"] = {}
+    for key, host in (("device_descriptors_only", None), ("with_host_descriptors", mdescs)):
+        ms, _ = timed(lambda: kvh.encode_chunks(w.kv, mdev, len(mdescs), w.stream_buf[:mtotal], w.status, descs=host))
+        out["encode_mixed_levels"][key] = {"ms": round(ms, 4), "hbm_gbps": round((2 * elements + mtotal) / ms / 1e6, 1)}
     runs, n_kept = kvh.keep_sinks_and_recent(N, 4, max(N // 4 - 4, 1))
     for level in LEVELS:
         descs, total = kvh.plan_chunks(l, c, n_kept, level)
@@ -774,6 +783,8 @@ def run_ours(args):
         for key in ("transcode", "token_dropping"):
             for r in extras[key]:
                 r["roofline_frac"] = round(r["hbm_gbps"] / peak, 4)
+        for r in extras["encode_mixed_levels"].values():
+            r["roofline_frac"] = round(r["hbm_gbps"] / peak, 4)
         out["extras"] = extras
     if single and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
@@ -792,6 +803,39 @@ def run_ours(args):
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_policy(args):
+    """Time the greedy policy (host C++) on synthetic entries: 16 stored forms per entry (4 levels x 4
+    kept fractions of the tokens), sizes from the library's own size arithmetic for the 8B shape,
+    capacity an eighth of the full-quality total.  One host core; no GPU work."""
+    import paper_2509_00105_b200 as kvh
+    n = args.policy_entries
+    l, c = workloads.LLAMA8B_8K.n_layers, 1024
+    rng = np.random.default_rng(7)
+    freq = 10.0 / (rng.permutation(n) + 1.0)
+    tokens = np.exp(rng.uniform(np.log(workloads.BATCH_MIN_TOKENS), np.log(workloads.BATCH_MAX_TOKENS), n)).astype(np.int64)
+    forms = [(level, keep) for keep in (1.0, 0.5, 0.25, 0.125) for level in range(4)]
+    chunk = {k: np.array([0] + [kvh.level_bytes(k, l, c, t) for t in range(1, 257)], dtype=np.int64) for k in range(4)}
+    sens_q, sens_d = 0.02 + 0.25 * rng.random(n), 0.05 + 0.9 * rng.random(n)
+    options = np.empty(n * len(forms), dtype=kvh.OPTION_DTYPE)
+    size_f, quality_f = options.dtype.names[:2]
+    for j, (level, keep) in enumerate(forms):
+        kept = np.maximum(1, (tokens * keep).astype(np.int64))
+        options[size_f][j::len(forms)] = (kept // 256) * chunk[level][256] + chunk[level][kept % 256]
+        options[quality_f][j::len(forms)] = np.maximum(0.0, (1 - sens_q * (level / 3.0) ** 2) * (1 - sens_d * ((1 - keep) / 0.875) ** 1.5))
+    begin = np.arange(0, n * len(forms) + 1, len(forms), dtype=np.int32)
+    capacity = int(options[size_f][0::len(forms)].sum() // 8)
+    times = []
+    for _ in range(max(1, min(args.steps or 3, 5))):
+        t = time.perf_counter()
+        choice, used, total = kvh.policy_assign(freq, options, begin, 2.0, 25e9, capacity)
+        times.append(time.perf_counter() - t)
+    assert used <= capacity
+    print(json.dumps({"metric": "policy entries/s (host, one core)", "value": n / min(times), "unit": "entries/s", "entries": n,
+                      "options_per_entry": len(forms), "seconds": round(min(times), 4), "us_per_entry": round(min(times) / n * 1e6, 3),
+                      "capacity_bytes": capacity, "used_bytes": int(used), "stored_entries": int((choice >= 0).sum()),
+                      "data": "synthetic"}))
 
 
 def free_port() -> int:
@@ -817,6 +861,10 @@ def main():
     ap.add_argument("--variant", choices=["default", "static"], default="default",
                     help="library build: 'static' walks tiles with a fixed stride (scheduling comparison)")
     ap.add_argument("--tokens", type=int, default=0, help="shorten the context (profiling only; not a bench line)")
+    ap.add_argument("--shape", default="", metavar="L,C,N",
+                    help="a single context of L layers, C channels, N tokens instead of a named workload (other row widths)")
+    ap.add_argument("--policy-entries", type=int, default=0,
+                    help="time the policy (host code) on this many synthetic entries instead of the codec, and exit")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--stat-launches", type=int, default=50, help="launches per level and direction in level_stats; 0 skips")
     ap.add_argument("--extras-reps", type=int, default=20, help="launches per transcode pair / token-dropping level in extras")
@@ -828,6 +876,15 @@ def main():
     if args.print_source_digest:
         print(kernel_source_digest())
         return
+    if args.policy_entries > 0:
+        run_policy(args)
+        return
+    if args.shape:
+        l, c, n = (int(x) for x in args.shape.split(","))
+        name = f"custom-l{l}-c{c}-n{n}"
+        SHAPES[name] = workloads.Shape(name, l, c, n)
+        WORKLOAD_NAMES.append(name)
+        args.workload = name
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(relaunch_as_ranks(args.gpus))
     if args.steps is None:
