@@ -1,13 +1,13 @@
 // Persistent, TMA-fed decode kernel (pages of >= 8 tokens; rows of up to 1024 channels, or wider
 // rows that divide into equal column blocks, which are fed with one bulk copy per row).
 //
-// One CTA (or a few) per SM loops over work units.  A producer warp walks the CTA's share of
-// (chunk, layer, K|V, 32-token tile) tiles, resolves descriptors and page ids, and streams each
-// unit's codes and group metadata from HBM into a ring of shared-memory stages with 1-D bulk
-// async copies (cp.async.bulk, completion counted on an mbarrier).  Eight consumer warps unpack,
-// dequantise and write full 16-byte vectors of page rows.  Copies for the next stages are always
-// in flight while the current one is being expanded, so HBM latency is off the critical path and
-// the kernel runs at the speed of its writes (2 of the (b+1)/8 + 2 bytes moved per element).
+// Three CTAs per SM loop over work units.  A producer warp walks the CTA's share of
+// (layer, K|V, chunk, 32-token tile) tiles, resolves descriptors and page ids, and streams each
+// unit's codes and group metadata from HBM into shared-memory stages with 1-D bulk async copies
+// (cp.async.bulk, completion counted on an mbarrier).  Eight consumer warps unpack, dequantise and
+// write full 16-byte vectors of page rows, row step by row step in lockstep.  Copies for the next
+// units are always in flight while the current one is being expanded, and the kernel runs at the
+// speed of its writes (2 of the (b+1)/8 + 2 bytes moved per element).
 //
 // A unit is a 32-token tile of a quantised plane (32*c*b/8 bytes of codes + 4*c bytes of metadata)
 // or one 16-token half of a raw bf16 tile (32*c bytes).  Rows of at most 512 channels would leave

@@ -7,13 +7,14 @@
 // (b_m + 1)/8 bytes and writes (b_n + 1)/8 bytes; a decode into a bf16 buffer followed by an encode
 // would move 4 more.
 //
-// Structure: the encode kernel's pipeline (3 shared-memory stages fed by 1-D bulk copies, tiles
+// Structure: the encode kernel's pipeline (shared-memory stages fed by 1-D bulk copies, tiles
 // handed out through cluster launch control, 8 consumer warps) with the decode kernel's unpacking
 // in front.  A level-0 source is the encoder itself reading the chunk's raw rows.  From a
 // quantised source the new range of every group follows from its old metadata (tc_new_meta), so a
 // K thread walks the rows of its 4 channels and a V thread its groups, one at a time: dequantise,
-// round to bf16, quantise again, store.  Such instances need few registers and small stages and
-// run two CTAs per SM.
+// round to bf16, quantise again, store.  Such instances need few registers and two small stages
+// and run three CTAs per SM.  They move about one byte per element and are bound by instruction
+// issue, not by memory.
 #pragma once
 
 #include "kvh_async.cuh"
@@ -242,7 +243,7 @@ __device__ __forceinline__ void tc_dispatch(const TcUnit &u, const uint8_t *st, 
 
 // sched as in the encode kernel.  One CTA per SM: 8 consumer warps and a producer warp.
 // Bytes of a stage: a raw tile (64 KiB at c = 1024) when the source may be level 0, else codes of at
-// most 8 bits plus metadata (36 KiB), which leaves room for two CTAs per SM.
+// most 8 bits plus metadata (36 KiB); two of those per CTA leave room for three CTAs per SM.
 template <int LIN>
 __host__ __device__ constexpr uint32_t tc_stage_bytes() { return LIN >= 1 ? 36u * 1024u : kEncStageBytes; }
 // Stages per CTA: two of them leave room for three CTAs per SM when the source is quantised.

@@ -219,6 +219,31 @@ def test_out_of_range_page_is_skipped_and_reported(kvh):
     assert np.array_equal(to_np16(flat), want_pool)
 
 
+@pytest.mark.parametrize("level", [0, 1, 2, 3])
+def test_out_of_range_pages_in_whole_tiles_at_the_compiled_in_width(kvh, level):
+    """Rows of 1024 channels and whole tiles take the unrolled consumers whose warps step through a
+    tile's rows behind a named barrier.  A page id outside the pool must make exactly the threads
+    that own its rows skip their stores: every other page is written, nothing else is touched, the
+    status says so, and every thread still reaches every barrier (the launch ends)."""
+    l, c, N = 2, 1024, 512
+    kv = workloads.make_kv(l, N, c, seed=80 + level, device="cuda")
+    got, _ = kvh.encode(kv, level)
+    want, offsets = oracle.encode_context(to_np16(kv), level)
+    assert np.array_equal(got.cpu().numpy(), want)
+    num_pages = 40
+    ids = workloads.shuffled_page_table(32, num_pages, seed=81).numpy().copy()
+    ids[[0, 5, 17, 31]] = [num_pages, -1, 1 << 30, num_pages + 7]      # first page of a tile, second page, both chunks
+    descs, _ = kvh.plan_chunks(l, c, N, level)
+    flat, view, strides = sentinel_pool(l, num_pages, c, pad=(128, 64, 32))
+    status = new_status()
+    kvh.decode_batch(got, kvh.descs_to_tensor(descs, "cuda"), len(descs), torch.from_numpy(ids).cuda(), kvh.Pool(view), status)
+    torch.cuda.synchronize()
+    want_pool, skipped = oracle_pool(flat.numel(), strides, want, offsets, [256, 256], [level, level], l, c, ids, num_pages)
+    assert skipped == 4 * 16 * l * 2
+    assert status.item() == 6
+    assert np.array_equal(to_np16(flat), want_pool)
+
+
 def test_bad_descriptors_are_skipped_and_reported(kvh):
     l, c, N = 1, 64, 512
     kv = workloads.make_kv(l, N, c, seed=9, device="cuda")
