@@ -60,6 +60,34 @@ __host__ __device__ __forceinline__ int ring_quanta(int c)
     const int q = (int)((72u * 1024u) / tma_quantum_bytes(c));
     return q < 6 ? 6 : (q > kMaxQuanta ? kMaxQuanta : q);
 }
+
+// The producer's book-keeping of the ring.  Units take their quanta at `head`, in order, as one
+// contiguous run: a unit that does not fit before the ring's end starts at 0 and takes the quanta
+// left before the end along with it (they come back when it does).  Quanta return in the order
+// they were taken (the consumers release units in order), so the free quanta are always the one
+// circular run from `head` to the oldest unit still held, and "enough free quanta" is all that has
+// to be checked.  With at least 6 quanta and units of at most 3, an empty ring takes any unit.
+struct QuantaRing {
+    int n_quanta, head, free_q;
+    __host__ __device__ explicit QuantaRing(int n) : n_quanta(n), head(0), free_q(n) {}
+    // quanta given up before the ring's end so that `need` of them are contiguous
+    __host__ __device__ int skipped(int need) const { return head + need > n_quanta ? n_quanta - head : 0; }
+    __host__ __device__ bool fits(int need) const { return free_q >= need + skipped(need); }
+    // Takes `need` contiguous quanta (fits(need) must hold): returns the index of the first and, in
+    // held, how many the unit keeps until it is given back (need + the ones skipped).
+    __host__ __device__ int take(int need, int &held)
+    {
+        const int skip = skipped(need);
+        if (skip) head = 0;
+        const int at = head;
+        head += need;
+        if (head == n_quanta) head = 0;
+        held = need + skip;
+        free_q -= held;
+        return at;
+    }
+    __host__ __device__ void give_back(int held) { free_q += held; }
+};
 __host__ __device__ __forceinline__ uint32_t round16(uint32_t x) { return (x + 15u) & ~15u; }
 
 // ---- dequantisation of 8 consecutive codes with few instructions per element ----------------
@@ -479,12 +507,11 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
         LayerLayout L = layer_layout(0, p.c, 1);
         uint32_t unit = 0;
         bool ok = true;
-        // The ring of quanta: units take their quanta at head_q, in order, never across the ring's end
-        // (the quanta left before the end are given up with the unit that did not fit there), and hand
-        // them back in the same order when the consumers release them.  tail is the oldest unit whose
-        // quanta have not been taken back; lane j remembers what the unit in slot j holds.
+        // tail is the oldest unit whose quanta have not been taken back; lane j remembers how many the
+        // unit in slot j holds
+        QuantaRing ring(n_quanta);
         uint32_t tail = 0;
-        int head_q = 0, free_q = n_quanta, slot_q = 0;
+        int slot_q = 0;
 
         // One unit.  Contiguous source (rows as wide as the plane): one copy of codes_bytes and one of
         // meta_bytes.  A column block of wider rows (row_stride != 0): lane r copies row r's codes_bytes
@@ -495,23 +522,19 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
                         uint32_t mrow_stride) -> bool {
             const int s = unit % kSlots;
             const int need = unit_quanta(bits);
-            const int pad = head_q + need > n_quanta ? n_quanta - head_q : 0;
-            while (unit - tail >= (uint32_t)kSlots || free_q < need + pad) {
-                if (tail == unit) return false;              // nothing left to take back: cannot happen (the ring holds any unit)
+            while (unit - tail >= (uint32_t)kSlots || !ring.fits(need)) {
+                if (tail == unit) return false;              // nothing left to take back: cannot happen (an empty ring holds any unit)
                 bool w = true;
                 if (lane == 0) w = mbar_wait(&empty_bar[tail % kSlots], (tail / kSlots) & 1, &abort_flag);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 if (!w) return false;
-                free_q += __shfl_sync(0xffffffffu, slot_q, tail % kSlots);
+                ring.give_back(__shfl_sync(0xffffffffu, slot_q, tail % kSlots));
                 ++tail;
             }
-            if (pad) head_q = 0;
-            const uint32_t st_off = (uint32_t)head_q * quantum;
+            int held;
+            const uint32_t st_off = (uint32_t)ring.take(need, held) * quantum;
             const uint32_t meta_off = 4u * (uint32_t)(bits == 16 ? 8 : bits) * p.bw * tpu;   // behind a tile's codes
-            head_q += need;
-            if (head_q == n_quanta) head_q = 0;
-            free_q -= need + pad;
-            if (lane == s) slot_q = need + pad;
+            if (lane == s) slot_q = held;
             const int pidx = row0 >> p.page_shift;
             int32_t pg[4];
 #pragma unroll

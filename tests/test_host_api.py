@@ -64,6 +64,7 @@ def test_build_variants_export_the_same_abi(kvh):
     with pytest.raises(ValueError):
         kvh.variant("nonesuch")
     assert hasattr(ctypes.CDLL(str(libs["selftest"])), "kvh_selftest_bounded_wait")
+    assert hasattr(ctypes.CDLL(str(libs["selftest"])), "kvh_selftest_quanta_ring")
 
 
 def test_versions_and_level_info(kvh):
@@ -237,3 +238,23 @@ def test_page_table_check(kvh):
     u = t.copy(); u[300] = u[12]
     assert kvh.check_page_table(u, 600) == (1, 300)
     assert kvh.check_page_table(np.zeros(0, dtype=np.int32), 5) == (0, -1)
+
+
+def test_ring_of_stage_quanta_never_overlaps_and_never_stalls_empty():
+    """The decode kernel cuts its shared-memory stages from a ring of quanta (1 to 3 per unit by
+    level, contiguous, taken and given back in order).  The producer's book-keeping is host/device
+    code; a test-only entry point (host code, no GPU) drives it with seeded sequences of unit sizes
+    against an occupancy map: a unit's quanta must be free when it gets them, lie inside the ring and
+    all come back, and an empty ring must take any unit."""
+    from paper_2509_00105_b200 import _build
+    L = ctypes.CDLL(str(_build.build(variant="selftest")))
+    L.kvh_selftest_quanta_ring.restype = ctypes.c_int64
+    L.kvh_selftest_quanta_ring.argtypes = [ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.POINTER(ctypes.c_int)]
+    most = ctypes.c_int(0)
+    for n_quanta in (6, 7, 9, 12, 18, 24):                    # 6: rows of 1024 channels; more: narrower rows
+        for seed in range(5):
+            assert L.kvh_selftest_quanta_ring(n_quanta, 200_000, seed, ctypes.byref(most)) == 0, (n_quanta, seed)
+            assert 2 <= most.value <= 8
+    assert most.value == 8                                     # 24 quanta: the 8 unit slots are the limit
+    assert L.kvh_selftest_quanta_ring(5, 10, 0, None) < 0 and L.kvh_selftest_quanta_ring(25, 10, 0, None) < 0
+    assert L.kvh_selftest_quanta_ring(6, 0, 0, ctypes.byref(most)) == 0
