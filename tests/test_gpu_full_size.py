@@ -238,3 +238,68 @@ def test_batched_mixed_level_load_at_scale(kvh):
     direct.decode_batch(blob, all_descs_dev, len(all_descs), table, direct.Pool(pool.tensor), status)
     assert status.item() == 0
     assert plane_checksums(pool) == sums
+
+
+def test_transcode_at_full_size_equals_decode_then_encode(kvh):
+    """The benchmark's transcoding launches (70B shape, 32,768 tokens), every pair of levels, whole
+    buffers: transcoding a stored context must give, byte for byte, what encoding at the new level
+    gives from the pages the old stream decodes to (the definition of the operation; both of those
+    paths are checked against the oracle above), and chunks spread over the launch must equal the
+    oracle's transcoding of the same stored bytes."""
+    s = workloads.LLAMA70B_32K
+    l, c, N = s.n_layers, s.n_channels, s.n_tokens
+    kv = workloads.make_kv(l, N, c, seed=4100, device="cuda")
+    n_pages = workloads.n_pages(N)
+    table = torch.arange(n_pages, dtype=torch.int32, device="cuda")          # identity: the pool is laid out like kv
+    pool = kvh.Pool.allocate(l, n_pages, c)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    plans = {k: kvh.plan_chunks(l, c, N, k) for k in range(4)}
+    devs = {k: kvh.descs_to_tensor(plans[k][0], "cuda") for k in range(4)}
+    n_chunks = len(plans[0][0])
+    sample = spread(n_chunks, 32)
+    for lin in (0, 1, 2):
+        src, _ = kvh.encode(kv, lin, dev_status=status)
+        pool.tensor.view(torch.int16).fill_(SENTINEL)
+        kvh.decode_batch(src, devs[lin], n_chunks, table, pool, status)
+        decoded = pool.tensor.view(l, 2, N, c)
+        for lout in range(lin + 1, 4):
+            want, total = kvh.encode(decoded, lout, dev_status=status)
+            got = torch.full((total + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+            kvh.transcode(src, devs[lin], got[:total], devs[lout], n_chunks, l, c, lin, lout, dev_status=status)
+            assert status.item() == 0
+            assert torch.equal(got[:total], want), f"transcode {lin}->{lout} differs from decode + encode"
+            assert bool((got[total:] == 0xAB).all())
+            if lin > 0:                                  # from level 0 the operation is the encoder itself
+
+                def one(i):
+                    a, b = int(plans[lin][0]["stream_off"][i]), int(plans[lout][0]["stream_off"][i])
+                    size_in = oracle.level_bytes(lin, l, c, 256)
+                    size_out = oracle.level_bytes(lout, l, c, 256)
+                    ref = oracle.transcode_chunk(src[a:a + size_in].cpu().numpy(), lin, lout, l, c, 256)
+                    assert np.array_equal(got[b:b + size_out].cpu().numpy(), ref), f"chunk {i}, {lin}->{lout}"
+
+                for i in sample[::3]:
+                    one(i)
+            del want, got
+        del src
+
+
+def test_token_dropping_at_full_size(kvh):
+    """The benchmark's token-dropping launches (70B shape, 4 sink tokens and a recent window, a quarter
+    of the context kept) at every level, whole buffers: encoding the kept runs must give, byte for
+    byte, the encoding of the compacted tensor (the definition of the operation)."""
+    s = workloads.LLAMA70B_32K
+    l, c, N = s.n_layers, s.n_channels, s.n_tokens
+    kv = workloads.make_kv(l, N, c, seed=4200, device="cuda")
+    runs, n_kept = kvh.keep_sinks_and_recent(N, 4, N // 4 - 4)
+    assert n_kept == N // 4 and len(runs) == 2
+    compact = torch.cat([kv[:, :, int(r["first"]):int(r["first"]) + int(r["count"])] for r in runs], dim=2).contiguous()
+    assert compact.shape[2] == n_kept
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for level in (0, 1, 2, 3):
+        want, total = kvh.encode(compact, level, dev_status=status)
+        got = torch.full((total + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+        kvh.encode_kept(kv, runs, None, workloads.n_chunks(n_kept), got[:total], status, level=level)
+        assert status.item() == 0
+        assert torch.equal(got[:total], want), f"kept-run encoding differs from the compacted encoding at level {level}"
+        assert bool((got[total:] == 0xAB).all())
