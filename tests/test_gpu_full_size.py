@@ -303,3 +303,47 @@ def test_token_dropping_at_full_size(kvh):
         assert status.item() == 0
         assert torch.equal(got[:total], want), f"kept-run encoding differs from the compacted encoding at level {level}"
         assert bool((got[total:] == 0xAB).all())
+
+
+def test_host_tier_at_full_size_with_a_level_per_chunk(kvh):
+    """The benchmark's end-to-end path at its full size (70B shape, 32,768 tokens), here with a random
+    level per chunk so that slices mix levels: what kvh_store_host leaves in pinned host memory must be,
+    byte for byte, what kvh_encode_chunks writes on the device, and what kvh_load_host decodes from
+    there must be, element for element, what one batched decode of the device copy gives (both of
+    those are checked against the oracle above)."""
+    s = workloads.LLAMA70B_32K
+    l, c, N = s.n_layers, s.n_channels, s.n_tokens
+    kv = workloads.make_kv(l, N, c, seed=4300, device="cuda")
+    levels = workloads.chunk_levels(workloads.n_chunks(N), 4, seed=4301)
+    descs, total = kvh.plan_chunks(l, c, N, levels)
+    descs_dev = kvh.descs_to_tensor(descs, "cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    host_status = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    copy_stream = torch.cuda.Stream()
+    want_stream = torch.empty(total, dtype=torch.uint8, device="cuda")
+    kvh.encode_chunks(kv, descs_dev, len(descs), want_stream, status, descs=descs)
+    n_pages = workloads.n_pages(N)
+    table = workloads.shuffled_page_table(n_pages, n_pages + 32, seed=4302).cuda()
+    want_pool = kvh.Pool.allocate(l, n_pages + 32, c)
+    want_pool.tensor.view(torch.int16).fill_(SENTINEL)
+    kvh.decode_batch(want_stream, descs_dev, len(descs), table, want_pool, status)
+    assert status.item() == 0
+
+    staging = torch.full((total,), 0x55, dtype=torch.uint8, device="cuda")
+    host = torch.full((total,), 0x66, dtype=torch.uint8).pin_memory()
+    kvh.store_host(kv, descs, descs_dev, staging, host, status, host_status, copy_stream)
+    torch.cuda.current_stream().synchronize()
+    assert host_status.item() == 0
+    back = torch.empty_like(want_stream)
+    back.copy_(host)
+    assert torch.equal(back, want_stream), "the stored form in host memory differs from the device encoding"
+    del back, kv
+
+    staging.fill_(0x77)
+    pool = kvh.Pool.allocate(l, n_pages + 32, c)
+    pool.tensor.view(torch.int16).fill_(SENTINEL)
+    host_status.fill_(-1)
+    kvh.load_host(host, staging, descs, descs_dev, table, pool, status, host_status, copy_stream)
+    torch.cuda.synchronize()
+    assert host_status.item() == 0
+    assert torch.equal(pool.tensor.view(torch.int16), want_pool.tensor.view(torch.int16))
