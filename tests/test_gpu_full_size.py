@@ -153,6 +153,17 @@ def test_wide_rows_llama2_7b_shape(kvh):
     run_context(kvh, s, seed=7000, levels=(0, 1, 2, 3), sample=[0, 7, 15])
 
 
+@pytest.mark.parametrize("c", [256, 768, 1280])
+def test_other_row_widths_at_scale(kvh, c):
+    """Rows that are not 1024 channels wide take other routes through the same kernels: 2 KV heads
+    (256 channels: four tiles per work unit), 6 heads (768: the general consumers, 2-D boxes in the
+    encoder) and 10 heads (1280: two column blocks of 640, one copy per row).  16 layers x 16,384
+    tokens each: thousands of units per launch, dynamic hand-out, every level; sampled chunks against
+    the oracle and whole buffers against the other kernel family."""
+    s = workloads.Shape(f"rows-{c}", 16, c, 16384)
+    run_context(kvh, s, seed=7100 + c, levels=(0, 1, 2, 3), sample=spread(workloads.n_chunks(s.n_tokens), 16))
+
+
 def plane_checksums(pool):
     """Two position-dependent 64-bit sums per (layer, K|V) plane (wrap-around arithmetic)."""
     out = []
