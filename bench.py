@@ -75,9 +75,9 @@ WORKLOAD_NAMES = ["tiny", "llama3-8b-8k", BATCH, "llama3-70b-32k", "llama3-8b-12
 # has changed, `traffic` is reported as null until the capture is repeated.
 TRAFFIC = {
     "captured": "2026-11-28",
-    "source_digest": "8d48dc22d17c57a6",
-    "decode": {0: 0.9804, 1: 0.9726, 2: 0.9665, 3: 0.9629},
-    "encode": {0: 0.9792, 1: 0.9798, 2: 0.9872, 3: 0.9919},
+    "source_digest": "ca5950608c05f5a8",
+    "decode": {0: 0.9801, 1: 0.9724, 2: 0.9673, 3: 0.9630},
+    "encode": {0: 0.9792, 1: 0.9795, 2: 0.9865, 3: 0.9919},
     # executed thread instructions per element of the transcoding instances whose source is quantised
     # (smsp__inst_executed.sum x 32 / elements of the same capture): these are bound by instruction
     # issue, not by memory

@@ -588,11 +588,21 @@ __global__ void __launch_bounds__(kTmaThreads, 3) decode_tma_kernel(const Decode
             // Order of the tiles: a chunk's tiles, then the chunks, then the (layer, K|V) planes.  CTAs that
             // run side by side thus write into one plane of the pool (pages scattered over 64 MiB, not over
             // the whole pool: the same few translations serve every SM) and read from neighbouring chunks.
+            // Rows cut into column blocks keep the order that finishes a chunk's planes first: their producer
+            // issues a copy per row and has no time to spare for a new descriptor at every unit (measured:
+            // 3-9 % slower plane by plane at 1280, 1536 and 4096 channels).
             const uint32_t t2 = row_tile / units;
-            const int chunk = (int)(t2 % (uint32_t)n_chunks);
-            const uint32_t plane_id = t2 / (uint32_t)n_chunks;
-            const int kv = (int)(plane_id & 1);
-            const int layer = (int)(plane_id >> 1);
+            int chunk, kv, layer;
+            if (nb == 1) {
+                chunk = (int)(t2 % (uint32_t)n_chunks);
+                const uint32_t plane_id = t2 / (uint32_t)n_chunks;
+                kv = (int)(plane_id & 1);
+                layer = (int)(plane_id >> 1);
+            } else {
+                kv = (int)(t2 & 1);
+                layer = (int)((t2 >> 1) % (uint32_t)p.l);
+                chunk = (int)((t2 >> 1) / (uint32_t)p.l);
+            }
             if (chunk != cur_chunk) {
                 cur_chunk = chunk;
                 if (p.descs) d = p.descs[chunk];
